@@ -1,0 +1,303 @@
+// Host side of the C ABI declared in include/tcu_scan.h: argument checks, workspace
+// sizing, TMA tensor-map encoding, variant dispatch, launch and bookkeeping.
+#include "tcu_scan.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstring>
+#include <mutex>
+
+#include "tcu_scan_kernel.cuh"
+
+namespace {
+
+using namespace tcu;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+std::mutex g_stats_mutex;
+tcu_scan_stats_t g_stats;
+bool g_have_stats = false;
+
+int elem_bytes(tcu_dtype_t dt) { return dt == TCU_I8_I32 ? 1 : 2; }
+bool valid_dtype(int dt) { return dt == TCU_I8_I32 || dt == TCU_F16_F32 || dt == TCU_BF16_F32; }
+bool valid_s(int s) { return s == 16 || s == 64 || s == 128; }
+
+uint64_t tiles_for(uint64_t rows, uint64_t cols) {
+    uint64_t rows128 = cols / kTileCols;                       // full 128-element rows of one scan
+    uint64_t per = (rows128 + kTileRows - 1) / kTileRows;      // tiles of one scan
+    return rows * per;
+}
+
+uint32_t floor_log(uint64_t n, uint64_t s) {
+    uint32_t k = 0;
+    uint64_t p = s;
+    while (p <= n) {
+        ++k;
+        if (p > n / s) break;
+        p *= s;
+    }
+    return k;
+}
+
+struct Shape {
+    uint64_t rows, cols;
+};
+
+template <bool IS_INT, int S, bool EXCL>
+cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
+    static std::atomic<int> configured{-1};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (configured.load() != dev) {
+        cudaError_t e = cudaFuncSetAttribute(tcu_scan_kernel<IS_INT, S, EXCL>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+        if (e != cudaSuccess) return e;
+        configured.store(dev);
+    }
+    tcu_scan_kernel<IS_INT, S, EXCL><<<grid, kThreads, smem, stream>>>(prm);
+    return cudaGetLastError();
+}
+
+template <bool IS_INT, bool EXCL>
+cudaError_t dispatch_s(int s, const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
+    switch (s) {
+        case 16: return launch_main<IS_INT, 16, EXCL>(prm, grid, smem, stream);
+        case 64: return launch_main<IS_INT, 64, EXCL>(prm, grid, smem, stream);
+        default: return launch_main<IS_INT, 128, EXCL>(prm, grid, smem, stream);
+    }
+}
+
+int sm_count() {
+    static std::atomic<int> cached{0};
+    int v = cached.load();
+    if (v > 0) return v;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    cached.store(v);
+    return v;
+}
+
+bool overlaps(const void *a, size_t an, const void *b, size_t bn) {
+    auto pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b);
+    return pa < pb + bn && pb < pa + an;
+}
+
+tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
+                       bool exclusive, bool level0, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    if (!valid_dtype(dt) || !valid_s(s)) return (s > 0 && valid_dtype(dt)) ? TCU_ERR_UNSUPPORTED : TCU_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return TCU_OK;
+    if (!d_in || !d_out) return TCU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_in) & 15) || (reinterpret_cast<uintptr_t>(d_out) & 15)) return TCU_ERR_INVALID_ARG;
+    const int eb = elem_bytes(dt);
+    if (rows > 1 && (cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
+    if (level0 && (cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
+    if (rows > (1ull << 31) || cols > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
+    const uint64_t total = uint64_t(rows) * cols;
+    if (overlaps(d_in, total * eb, d_out, total * 4)) return TCU_ERR_INVALID_ARG;
+    if (!d_ws) return TCU_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
+    if (ws_bytes < tcu_scan_workspace_bytes(rows, cols, dt, s)) return TCU_ERR_WORKSPACE;
+
+    const uint64_t rows128 = cols / kTileCols;
+    const uint64_t tiles_per_row = (rows128 + kTileRows - 1) / kTileRows;
+    const uint64_t tiles = rows * tiles_per_row;
+    const uint32_t tail = uint32_t(cols % kTileCols);
+    if (tiles >= (1ull << 31)) return TCU_ERR_UNSUPPORTED;
+
+    const int per32 = 32 / eb;
+    const int seff = s > per32 ? s : per32;
+    const int b_atoms = (seff * eb + 127) / 128;
+    const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
+    const uint32_t stage_bytes = kTileElems * eb;
+    const size_t fixed = kConstOffset + b_bytes + size_t(kOutChunks) * kOutChunkBytes + 1024;  // + alignment slack
+    int in_stages = int((232448 - fixed) / stage_bytes);
+    if (in_stages > kMaxInStages) in_stages = kMaxInStages;
+    if (in_stages > 4 && eb == 2) in_stages = 4;
+    if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
+    const size_t smem = fixed + size_t(in_stages) * stage_bytes;
+
+    tcu_scan_stats_t st;
+    std::memset(&st, 0, sizeof(st));
+    st.rows = rows;
+    st.cols = cols;
+    st.s = s;
+    st.dtype = dt;
+    st.exclusive = exclusive;
+    st.variant = 0;
+    st.upper_level_path = 0;
+    st.tiles = tiles;
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32));
+    st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
+    // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
+    // scan over the tiles (absent for a single tile), carry add
+    st.levels_used = 1 + (s < kTileCols ? 1 : 0) + 1 + (tiles_per_row > 1 ? 1 : 0) + 1;
+    st.depth_bound = 2 * floor_log(cols, uint64_t(s));
+    st.in_stages = in_stages;
+    st.smem_bytes = uint32_t(smem);
+    st.tail_elements = tail;
+
+    if (tiles > 0) {
+        EncodeTiledFn encode = get_encode_fn();
+        if (!encode) return TCU_ERR_CUDA;
+        int sms = sm_count();
+        if (sms <= 0) return TCU_ERR_CUDA;
+        ScanParams prm;
+        std::memset(&prm, 0, sizeof(prm));
+        const cuuint64_t dims[3] = {cuuint64_t(kTileCols), cuuint64_t(rows128), cuuint64_t(rows)};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        // stride between scans: the row pitch for batched input; for a single array any multiple of
+        // 16 bytes will do (the coordinate is always 0), and n itself need not be one
+        const cuuint64_t pitch_elems = rows > 1 ? cuuint64_t(cols) : cuuint64_t(rows128) * kTileCols;
+        {
+            const cuuint64_t strides[2] = {cuuint64_t(kTileCols) * eb, pitch_elems * eb};
+            const cuuint32_t box[3] = {cuuint32_t(128 / eb), cuuint32_t(kTileRows), 1};
+            CUtensorMapDataType ty = dt == TCU_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                     : dt == TCU_F16_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                         : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+            CUresult r = encode(&prm.tmap_in, ty, 3, const_cast<void *>(d_in), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
+        }
+        {
+            const cuuint64_t strides[2] = {cuuint64_t(kTileCols) * 4, pitch_elems * 4};
+            const cuuint32_t box[3] = {32, cuuint32_t(kTileRows), 1};
+            CUtensorMapDataType ty = dt == TCU_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+            CUresult r = encode(&prm.tmap_out, ty, 3, d_out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
+        }
+        prm.ws = d_ws;
+        prm.tiles_total = uint32_t(tiles);
+        prm.tiles_per_row = uint32_t(tiles_per_row);
+        prm.in_stages = uint32_t(in_stages);
+        prm.b_bytes = b_bytes;
+        prm.dtype = uint32_t(dt);
+        prm.level0_only = level0 ? 1u : 0u;
+        // persistent grid: every CTA must be resident at once (the carry chain waits on
+        // lower-numbered tiles), so never more CTAs than SMs; one CTA fills an SM's shared memory
+        dim3 grid(unsigned(tiles < uint64_t(sms) ? tiles : uint64_t(sms)));
+        st.grid = grid.x;
+        cudaError_t e;
+        if (dt == TCU_I8_I32)
+            e = exclusive ? dispatch_s<true, true>(s, prm, grid, smem, stream) : dispatch_s<true, false>(s, prm, grid, smem, stream);
+        else
+            e = exclusive ? dispatch_s<false, true>(s, prm, grid, smem, stream) : dispatch_s<false, false>(s, prm, grid, smem, stream);
+        if (e != cudaSuccess) return TCU_ERR_CUDA;
+    }
+    if (tail > 0) {   // only reachable with rows == 1
+        const size_t start = size_t(rows128) * kTileCols;
+        if (dt == TCU_I8_I32) {
+            if (exclusive) tcu_scan_tail_kernel<true, true><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
+            else tcu_scan_tail_kernel<true, false><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
+        } else {
+            if (exclusive) tcu_scan_tail_kernel<false, true><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
+            else tcu_scan_tail_kernel<false, false><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
+        }
+        if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+    }
+    {
+        std::lock_guard<std::mutex> lk(g_stats_mutex);
+        g_stats = st;
+        g_have_stats = true;
+    }
+    return TCU_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s) {
+    (void)dt;
+    (void)s;
+    return size_t(kHeaderBytes) + 16 * size_t(tiles_for(rows, cols)) + 16;
+}
+
+tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    if (!d_ws || ws_bytes < size_t(kHeaderBytes)) return TCU_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
+    return cudaMemsetAsync(d_ws, 0, ws_bytes, stream) == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+}
+
+tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
+                                size_t ws_bytes, cudaStream_t stream) {
+    return scan_impl(d_in, d_out, 1, n, dt, s, false, false, d_ws, ws_bytes, stream);
+}
+
+tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
+                                size_t ws_bytes, cudaStream_t stream) {
+    return scan_impl(d_in, d_out, 1, n, dt, s, true, false, d_ws, ws_bytes, stream);
+}
+
+tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
+                              int exclusive, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    return scan_impl(d_in, d_out, rows, cols, dt, s, exclusive != 0, false, d_ws, ws_bytes, stream);
+}
+
+tcu_status_t tcu_scan_level0_debug(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
+                                   size_t ws_bytes, cudaStream_t stream) {
+    return scan_impl(d_in, d_out, 1, n, dt, s, false, true, d_ws, ws_bytes, stream);
+}
+
+tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t dt, int s, int exclusive, void *d_in,
+                           void *d_out, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    if (!valid_dtype(dt)) return TCU_ERR_INVALID_ARG;
+    if (n == 0) return TCU_OK;
+    if (!h_in || !h_out || !d_in || !d_out) return TCU_ERR_INVALID_ARG;
+    if (cudaMemcpyAsync(d_in, h_in, n * elem_bytes(dt), cudaMemcpyHostToDevice, stream) != cudaSuccess) return TCU_ERR_CUDA;
+    tcu_status_t st = scan_impl(d_in, d_out, 1, n, dt, s, exclusive != 0, false, d_ws, ws_bytes, stream);
+    if (st != TCU_OK) return st;
+    if (cudaMemcpyAsync(h_out, d_out, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TCU_ERR_CUDA;
+    return TCU_OK;
+}
+
+tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream) {
+    if (!d_ws) return TCU_ERR_WORKSPACE;
+    WsHeader h;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return TCU_ERR_CUDA;
+    if (cudaMemcpy(&h, d_ws, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return TCU_ERR_CUDA;
+    return h.error == 0 ? TCU_OK : TCU_ERR_TIMEOUT;
+}
+
+tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out) {
+    if (!out) return TCU_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_stats_mutex);
+    if (!g_have_stats) return TCU_ERR_INVALID_ARG;
+    *out = g_stats;
+    return TCU_OK;
+}
+
+const char *tcu_status_string(tcu_status_t st) {
+    switch (st) {
+        case TCU_OK: return "ok";
+        case TCU_ERR_INVALID_ARG: return "invalid argument";
+        case TCU_ERR_UNSUPPORTED: return "unsupported request";
+        case TCU_ERR_WORKSPACE: return "workspace missing or too small";
+        case TCU_ERR_CUDA: return "CUDA call failed";
+        case TCU_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

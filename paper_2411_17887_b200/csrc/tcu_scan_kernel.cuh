@@ -1,0 +1,650 @@
+// Single-pass tensor-core-unit scan for sm_100a: device code.
+//
+// One persistent CTA per SM walks 128 x 128-element tiles in increasing order.
+//   warp 0    TMA producer: cp.async.bulk.tensor loads of the tile into a shared-memory ring
+//   warp 1    MMA issuer:   tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into TMEM
+//             (Algorithm 1, up-sweep round t = 0: every length-s chunk becomes its local scan)
+//   warp 2    carry scan across tiles: decoupled look-back over per-tile records in global
+//             memory (Section 2.2 steps 2-3: totals of the segments, and their scan)
+//   warps 4-7 epilogue: pass 1 reads the chunk totals from TMEM and scans them along the
+//             row and across the 128 rows (up-sweep rounds t >= 1); pass 2 adds chunk, row and
+//             tile carries to every element on the vector ALUs (down-sweep; the paper's
+//             discussion section recommends a vector unit for this add), stages the result
+//             in swizzled shared memory and writes it with TMA stores.
+// Every wait is bounded; a wait that runs out records TCU_ERR_TIMEOUT in the workspace
+// header, and the CTA winds down (drains its copies, frees TMEM) instead of spinning.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tcu {
+
+constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM lanes
+constexpr int kTileCols = 128;          // elements per tile row
+constexpr int kTileElems = kTileRows * kTileCols;
+constexpr int kNumAcc = 4;              // TMEM accumulators (128 columns each, 512 in all)
+constexpr int kRunAhead = 2;            // tiles by which epilogue pass 1 leads pass 2
+constexpr int kOutChunks = 6;           // ring of 16 KB output staging buffers (32 columns x 128 rows)
+constexpr int kOutChunkBytes = 32 * 4 * kTileRows;
+constexpr int kMaxInStages = 6;
+constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
+constexpr int kThreads = 256;
+constexpr int kEpilogueThreads = 128;
+constexpr int kFirstEpilogueWarp = 4;
+
+// workspace: 256-byte header, then one 16-byte record per tile
+constexpr int kHeaderBytes = 256;
+constexpr uint32_t kStatusPartial = 1;    // record holds the tile's own total
+constexpr uint32_t kStatusInclusive = 2;  // record holds the sum of everything up to and including the tile
+struct WsHeader {
+    uint32_t epoch;      // launches completed on this workspace
+    uint32_t done;       // CTAs of the running launch that have finished
+    uint32_t error;      // tcu_status_t recorded by a bounded wait that ran out
+    uint32_t pad[61];
+};
+static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
+
+constexpr long long kSpinLimitCycles = 2000000000LL;   // about one second at B200 clocks
+
+struct alignas(64) ScanParams {
+    CUtensorMap tmap_in;      // (128, rows128, batch) view of the input, box 128 B x 128 rows
+    CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 128 rows
+    void *ws;
+    uint32_t tiles_total;     // all tiles of the launch
+    uint32_t tiles_per_row;   // tiles of one scan (carry chain restarts every tiles_per_row tiles)
+    uint32_t in_stages;       // depth of the input ring
+    uint32_t b_bytes;         // shared memory reserved for the constant operand
+    uint32_t dtype;           // tcu_dtype_t
+    uint32_t level0_only;     // debug: stop after the U_s product (no carries)
+};
+
+// shared-memory bookkeeping (lives at the 1024-aligned base of dynamic shared memory)
+struct SmemCtl {
+    uint64_t full[kMaxInStages];     // TMA -> MMA
+    uint64_t empty[kMaxInStages];    // MMA -> TMA
+    uint64_t acc_full[kNumAcc];      // MMA -> epilogue
+    uint64_t acc_empty[kNumAcc];     // epilogue -> MMA
+    uint64_t agg_ready[kNumAcc];     // epilogue pass 1 -> carry warp
+    uint64_t carry_ready[kNumAcc];   // carry warp -> epilogue pass 2
+    uint64_t agg_slot[kNumAcc];      // tile total (bits of a double, or a zero-extended uint32)
+    uint64_t carry_slot[kNumAcc];    // sum of all earlier tiles of the same scan
+    uint32_t warp_tot[2][4];         // cross-warp hop of the 128-row scan (double buffered)
+    uint32_t tmem_base;
+    uint32_t epoch;
+    volatile uint32_t abort_flag;
+};
+constexpr int kCtlBytes = 1024;
+static_assert(sizeof(SmemCtl) <= kCtlBytes, "control block too large");
+constexpr int kRowPrefBytes = kNumAcc * kTileRows * 4;
+constexpr int kConstOffset = kCtlBytes + kRowPrefBytes;   // 3072: 1024-aligned
+static_assert(kConstOffset % 1024 == 0, "operand regions must be 1024-byte aligned");
+
+// ------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// barrier over `threads` threads that also ORs a predicate; every caller gets the same answer
+__device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred) {
+    uint32_t res;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(res)
+        : "r"(uint32_t(pred)), "r"(id), "r"(threads)
+        : "memory");
+    return res != 0;
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+template <bool IS_INT>
+__device__ __forceinline__ void mma_issue(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    if (IS_INT) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+__device__ __forceinline__ uint32_t tmem_ld1(uint32_t taddr) {
+    uint32_t v;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v) : "r"(taddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void ld_record(const void *p, uint64_t &flag, uint64_t &val) {
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(flag), "=l"(val) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_record(void *p, uint64_t flag, uint64_t val) {
+    asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(flag), "l"(val) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// ------------------------------------------------------------------------------------ descriptors
+// Shared-memory matrix descriptor of tcgen05.mma for a K-major operand stored as rows of
+// 128 bytes with the 128-byte swizzle: start address >> 4 in bits [0,14), stride between
+// 8-row groups (1024 B) >> 4 in bits [32,46), descriptor version 1 in bits [46,48), swizzle
+// mode 2 (128 B) in bits [61,64).  The leading-dimension offset is not used by this layout.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFF);
+    d |= static_cast<uint64_t>(1) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+// Instruction descriptor: accumulator format in bits [4,6) (1 = fp32, 2 = int32), A / B
+// formats in bits [7,10) / [10,13) (f16 kinds: 0 = fp16, 1 = bf16; i8 kind: 1 = signed),
+// both operands K-major (bits 15, 16 clear), N >> 3 in bits [17,23), M >> 4 in bits [24,29).
+__device__ __forceinline__ uint32_t make_idesc(uint32_t dtype, uint32_t n) {
+    uint32_t cfmt = (dtype == 0) ? 2u : 1u;
+    uint32_t abfmt = (dtype == 0) ? 1u : (dtype == 2 ? 1u : 0u);
+    return (cfmt << 4) | (abfmt << 7) | (abfmt << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------ helpers
+struct Waiter {
+    SmemCtl *ctl;
+    WsHeader *hdr;
+    // Wait for the phase of `bar` with the given parity; false when the wait was given up.
+    __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+        if (mbar_try_wait(bar, parity)) return true;
+        long long t0 = clock64();
+        uint32_t spins = 0;
+        while (!mbar_try_wait(bar, parity)) {
+            if ((++spins & 0xFF) == 0) {
+                if (ctl->abort_flag) return false;
+                if (clock64() - t0 > kSpinLimitCycles) {
+                    ctl->abort_flag = 1;
+                    atomicExch(&hdr->error, 5u);
+                    return false;
+                }
+            }
+        }
+        return true;
+    }
+};
+
+template <bool IS_INT> struct CarryOps;
+template <> struct CarryOps<true> {
+    using T = uint32_t;
+    static __device__ __forceinline__ uint64_t enc(T v) { return v; }
+    static __device__ __forceinline__ T dec(uint64_t b) { return static_cast<uint32_t>(b); }
+};
+template <> struct CarryOps<false> {
+    using T = double;
+    static __device__ __forceinline__ uint64_t enc(T v) { return static_cast<uint64_t>(__double_as_longlong(v)); }
+    static __device__ __forceinline__ T dec(uint64_t b) { return __longlong_as_double(static_cast<long long>(b)); }
+};
+template <typename T>
+__device__ __forceinline__ T warp_sum(T v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// element arithmetic of the epilogue on raw 32-bit registers
+template <bool IS_INT>
+__device__ __forceinline__ uint32_t add32(uint32_t a, uint32_t b) {
+    if (IS_INT) return a + b;
+    return __float_as_uint(__uint_as_float(a) + __uint_as_float(b));
+}
+
+// ------------------------------------------------------------------------------------ kernel
+template <bool IS_INT, int S, bool EXCL>
+__global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_constant__ ScanParams p) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    constexpr int kElemBytes = IS_INT ? 1 : 2;
+    constexpr int kPer32B = 32 / kElemBytes;                 // K of one MMA instruction
+    constexpr int kSeff = (S > kPer32B) ? S : kPer32B;       // side of the block-diagonal constant I (x) U_s
+    constexpr int kSegs = kTileCols / kSeff;                 // MMA groups per tile row
+    constexpr int kKSteps = kSeff / kPer32B;                 // accumulating MMAs per group
+    constexpr int kStageBytes = kTileElems * kElemBytes;     // 16 KB (int8) or 32 KB (16-bit)
+    constexpr int kInAtoms = kStageBytes / kAtomBytes;
+    constexpr int kChunksPerRow = kTileCols / S;             // length-s chunks in a tile row
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem);
+    uint32_t *rowpref = reinterpret_cast<uint32_t *>(smem + kCtlBytes);
+    uint8_t *const_region = smem + kConstOffset;
+    uint8_t *in_ring = const_region + p.b_bytes;
+    uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
+
+    WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
+    uint8_t *records = reinterpret_cast<uint8_t *>(p.ws) + kHeaderBytes;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t num_in = p.in_stages;
+
+    // ---- set-up
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kMaxInStages; ++i) {
+            mbar_init(smem_u32(&ctl->full[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < kNumAcc; ++i) {
+            mbar_init(smem_u32(&ctl->acc_full[i]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[i]), kEpilogueThreads);
+            mbar_init(smem_u32(&ctl->agg_ready[i]), 1);
+            mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
+        }
+        ctl->abort_flag = 0;
+        ctl->epoch = ld_relaxed_u32(&hdr->epoch) + 1;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), 512);
+        tmem_relinquish();
+    }
+    // constant operand: row n of the K-major storage holds column n of I (x) U_s, i.e. ones at
+    // k <= n inside the same s-block (U_s is L_s transposed: X U_s = (L_s X^T)^T).
+    {
+        uint32_t *cz = reinterpret_cast<uint32_t *>(const_region);
+        for (uint32_t i = threadIdx.x; i < p.b_bytes / 4; i += kThreads) cz[i] = 0;
+        __syncthreads();
+        for (int e = threadIdx.x; e < kSeff * kSeff; e += kThreads) {
+            int n = e / kSeff, k = e % kSeff;
+            if ((n / S) == (k / S) && k <= n) {
+                int kb = k * kElemBytes;
+                int off = (kb >> 7) * kAtomBytes + n * 128 + ((((kb & 127) >> 4) ^ (n & 7)) << 4) + (kb & 15);
+                if (IS_INT) {
+                    const_region[off] = 1;
+                } else {
+                    *reinterpret_cast<uint16_t *>(const_region + off) = (p.dtype == 2) ? 0x3F80 : 0x3C00;
+                }
+            }
+        }
+        fence_proxy_async_smem();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const uint32_t tmem_base = ctl->tmem_base;
+    const uint32_t epoch = ctl->epoch;
+    Waiter w{ctl, hdr};
+
+    const uint32_t first_tile = blockIdx.x;
+    const uint32_t stride = gridDim.x;
+    const uint32_t my_tiles = (p.tiles_total > first_tile) ? (p.tiles_total - first_tile + stride - 1) / stride : 0;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t issued = 0;
+            for (uint32_t j = 0; j < my_tiles; ++j) {
+                uint32_t t = first_tile + j * stride;
+                uint32_t stage = j % num_in, u = j / num_in;
+                if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
+                uint32_t bar = smem_u32(&ctl->full[stage]);
+                mbar_expect_tx(bar, kStageBytes);
+                int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
+#pragma unroll
+                for (int a = 0; a < kInAtoms; ++a)
+                    tma_load_3d(smem_u32(in_ring + stage * kStageBytes + a * kAtomBytes), &p.tmap_in,
+                                a * (128 / kElemBytes), lt * kTileRows, scan_row, bar);
+                issued = j + 1;
+            }
+            if (ctl->abort_flag) {
+                // drain: loads already issued must land before the CTA may exit
+                uint32_t lo = issued > num_in ? issued - num_in : 0;
+                for (uint32_t j = lo; j < issued; ++j) {
+                    uint32_t bar = smem_u32(&ctl->full[j % num_in]);
+                    uint32_t par = (j / num_in) & 1;
+                    long long t0 = clock64();
+                    while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinLimitCycles) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(p.dtype, kSeff);
+            const uint32_t b_base = smem_u32(const_region);
+            for (uint32_t j = 0; j < my_tiles; ++j) {
+                uint32_t stage = j % num_in, u = j / num_in;
+                uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+                if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
+                tc_fence_after();
+                const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
+#pragma unroll
+                for (int g = 0; g < kSegs; ++g) {
+#pragma unroll
+                    for (int kk = 0; kk < kKSteps; ++kk) {
+                        int a_off = (g * kKSteps + kk) * 32;
+                        int b_off = kk * 32;
+                        uint64_t adesc = make_smem_desc(a_base + (a_off >> 7) * kAtomBytes + (a_off & 127));
+                        uint64_t bdesc = make_smem_desc(b_base + (b_off >> 7) * kAtomBytes + (b_off & 127));
+                        mma_issue<IS_INT>(tmem_base + slot * kTileCols + g * kSeff, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                    }
+                }
+                mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once the MMAs have read it
+                mma_commit(smem_u32(&ctl->acc_full[slot]));    // the accumulator is complete
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ cross-tile carry scan
+        for (uint32_t j = 0; j < my_tiles; ++j) {
+            uint32_t t = first_tile + j * stride;
+            uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+            if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[slot]), ua & 1))) break;
+            const CarryT agg = CO::dec(ctl->agg_slot[slot]);
+            const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
+            CarryT prefix = CarryT(0);
+            if (static_cast<int>(t) == t0) {
+                if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(agg));
+            } else {
+                if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusPartial, CO::enc(agg));
+                int pos = static_cast<int>(t) - 1;
+                bool gave_up = false;
+                while (true) {
+                    int idx = pos - lane;
+                    bool valid = idx >= t0;
+                    uint64_t flag = 0, val = 0;
+                    if (valid) {
+                        const void *rec = records + size_t(idx) * 16;
+                        ld_record(rec, flag, val);
+                        if (static_cast<uint32_t>(flag >> 2) != epoch) {
+                            long long c0 = clock64();
+                            uint32_t spins = 0;
+                            while (true) {
+                                ld_record(rec, flag, val);
+                                if (static_cast<uint32_t>(flag >> 2) == epoch) break;
+                                if ((++spins & 0x3F) == 0 && (ctl->abort_flag || clock64() - c0 > kSpinLimitCycles)) {
+                                    gave_up = true;
+                                    flag = kStatusInclusive;   // treat as a chain end so that the walk stops
+                                    val = 0;
+                                    break;
+                                }
+                            }
+                        }
+                    }
+                    bool incl = valid && ((flag & 3) == kStatusInclusive);
+                    unsigned m = __ballot_sync(0xffffffffu, incl);
+                    CarryT v = valid ? CO::dec(val) : CarryT(0);
+                    if (m) {
+                        int first = __ffs(m) - 1;              // nearest predecessor whose record is inclusive
+                        if (lane > first) v = CarryT(0);
+                        prefix += warp_sum(v);
+                        break;
+                    }
+                    prefix += warp_sum(v);
+                    pos -= 32;
+                    if (pos < t0) break;
+                }
+                if (__any_sync(0xffffffffu, gave_up)) {
+                    if (lane == 0) {
+                        ctl->abort_flag = 1;
+                        atomicExch(&hdr->error, 5u);
+                    }
+                }
+                // publish even after a give-up so that successors do not wait for this tile
+                if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
+            }
+            if (lane == 0) {
+                ctl->carry_slot[slot] = CO::enc(prefix);
+                mbar_arrive(smem_u32(&ctl->carry_ready[slot]));
+            }
+            __syncwarp();
+        }
+    } else if (warp >= kFirstEpilogueWarp) {
+        // ------------------------------------------------------------------ epilogue
+        const int r = threadIdx.x - kFirstEpilogueWarp * 32;        // tile row owned by this thread = TMEM lane
+        const int wq = r >> 5;
+        const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
+        const uint32_t out_base = smem_u32(out_ring);
+        const bool issuer = (r == 0);
+        uint32_t chunk_counter = 0;
+        bool dead = false;
+
+        for (uint32_t i = 0; i < my_tiles + kRunAhead && !dead; ++i) {
+            if (i < my_tiles) {
+                // ---- pass 1: totals of the row, scan over the 128 rows, tile total
+                const uint32_t j = i;
+                const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+                // a wait that ran out is voted on at the next barrier, so that all 128 threads leave together
+                const bool ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
+                tc_fence_after();
+                uint32_t tot[kChunksPerRow];
+#pragma unroll
+                for (int g = 0; g < kChunksPerRow; ++g) tot[g] = tmem_ld1(lane_base + slot * kTileCols + g * S + (S - 1));
+                tmem_ld_wait();
+                uint32_t rowtot = tot[0];
+#pragma unroll
+                for (int g = 1; g < kChunksPerRow; ++g) rowtot = add32<IS_INT>(rowtot, tot[g]);
+                uint32_t inc = rowtot;                                // inclusive scan across the warp's 32 rows
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    uint32_t up = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc = add32<IS_INT>(inc, up);
+                }
+                uint32_t exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                if (lane == 0) exc = 0;
+                const int pb = j & 1;
+                if (lane == 31) ctl->warp_tot[pb][wq] = inc;
+                if (named_barrier_or(1, kEpilogueThreads, !ok)) { dead = true; break; }
+                uint32_t w0 = ctl->warp_tot[pb][0], w1 = ctl->warp_tot[pb][1], w2 = ctl->warp_tot[pb][2], w3 = ctl->warp_tot[pb][3];
+                uint32_t before = 0;                                  // rows of the earlier warps
+                if (wq >= 1) before = w0;
+                if (wq >= 2) before = add32<IS_INT>(before, w1);
+                if (wq >= 3) before = add32<IS_INT>(before, w2);
+                rowpref[slot * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
+                if (issuer) {
+                    uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
+                    CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
+                    ctl->agg_slot[slot] = CO::enc(a);
+                    mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
+                }
+            }
+            if (i >= kRunAhead) {
+                // ---- pass 2: add the carries, stage, store
+                const uint32_t j = i - kRunAhead;
+                const uint32_t t = first_tile + j * stride;
+                const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+                const bool ok = w.wait(smem_u32(&ctl->carry_ready[slot]), ua & 1);
+                const int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
+                uint32_t base;                                        // sum of everything before this row
+                {
+                    CarryT carry = CO::dec(ctl->carry_slot[slot]);
+                    uint32_t rp = rowpref[slot * kTileRows + r];
+                    if (IS_INT) base = uint32_t(carry) + rp;
+                    else base = __float_as_uint(static_cast<float>(double(carry) + double(__uint_as_float(rp))));
+                }
+                const bool level0 = p.level0_only != 0;
+                if (level0) base = 0;
+                uint32_t run = base;                                  // sum of everything before the current chunk
+                uint32_t prev = base;                                 // value of the element to the left (exclusive form)
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t d[32];
+                    tmem_ld32(lane_base + slot * kTileCols + q * 32, d);
+                    tmem_ld_wait();
+                    uint32_t o[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        uint32_t v = add32<IS_INT>(d[c], run);
+                        o[c] = EXCL ? prev : v;
+                        prev = v;
+                        const bool chunk_end = (S <= 32) ? (((c + 1) % S) == 0) : (c == 31 && (((q + 1) * 32) % S) == 0);
+                        if (chunk_end && !level0) run = v;            // end of a chunk: its total joins the carry
+                    }
+                    if (level0 && EXCL) {                             // not a meaningful combination; keep it defined
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) o[c] = d[c];
+                    }
+                    const uint32_t buf = out_base + (chunk_counter % kOutChunks) * kOutChunkBytes + r * 128;
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4)
+                        st_shared_v4(buf + ((c4 ^ (r & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
+                    fence_proxy_async_smem();
+                    if (issuer) bulk_wait_read<kOutChunks - 2>();      // the buffer of the next chunk has been drained
+                    if (named_barrier_or(1, kEpilogueThreads, !ok)) { dead = true; break; }
+                    if (issuer) {
+                        tma_store_3d(&p.tmap_out, out_base + (chunk_counter % kOutChunks) * kOutChunkBytes, q * 32, lt * kTileRows, scan_row);
+                        bulk_commit();
+                    }
+                    ++chunk_counter;
+                }
+                if (dead) break;
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
+            }
+        }
+        if (issuer) bulk_wait_all();
+    }
+
+    // ---- tear-down
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+    if (threadIdx.x == 0) {
+        __threadfence();
+        uint32_t old = atomicAdd(&hdr->done, 1u);
+        if (old == gridDim.x - 1) {          // last CTA: the launch is over, open the next epoch
+            hdr->done = 0;
+            __threadfence();
+            hdr->epoch = epoch;
+        }
+    }
+}
+
+// Tail of a single-array scan: the n % 128 elements after the last full 128-element row.
+// Runs after the main kernel on the same stream; the carry is the inclusive record of the
+// last tile (or nothing when there is no full row).
+template <bool IS_INT, bool EXCL>
+__global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start, uint32_t count, const void *ws,
+                                     uint32_t tiles, uint32_t dtype) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    __shared__ CarryT warp_tot[4];
+    const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
+    CarryT carry = CarryT(0);
+    if (tiles > 0) {
+        uint64_t flag, val;
+        ld_record(reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes + size_t(tiles - 1) * 16, flag, val);
+        carry = CO::dec(val);
+    }
+    CarryT x = CarryT(0);
+    if (tid < int(count)) {
+        if (IS_INT) {
+            x = CarryT(int32_t(reinterpret_cast<const int8_t *>(in)[start + tid]));
+        } else {
+            uint16_t b = reinterpret_cast<const uint16_t *>(in)[start + tid];
+            float f = (dtype == 2) ? __uint_as_float(uint32_t(b) << 16) : __half2float(__ushort_as_half(b));
+            x = CarryT(f);
+        }
+    }
+    CarryT inc = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        CarryT up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+    }
+    if (lane == 31) warp_tot[wq] = inc;
+    __syncthreads();
+    CarryT before = carry;
+    for (int k = 0; k < wq; ++k) before += warp_tot[k];
+    CarryT y = before + (EXCL ? (inc - x) : inc);
+    if (EXCL && !IS_INT) {   // avoid the subtraction's rounding: rebuild the exclusive value from the neighbour
+        CarryT left = __shfl_up_sync(0xffffffffu, inc, 1);
+        y = before + (lane == 0 ? CarryT(0) : left);
+    }
+    if (tid < int(count)) {
+        if (IS_INT) reinterpret_cast<uint32_t *>(out)[start + tid] = uint32_t(y);
+        else reinterpret_cast<float *>(out)[start + tid] = float(y);
+    }
+}
+
+}  // namespace tcu

@@ -1,0 +1,75 @@
+"""GPU parity at the full sizes of the five build configurations (plus the fp16 run of the
+headline size), in the launch configuration the benchmark times.  The oracle is evaluated
+piecewise (carry handed from piece to piece) so that host memory stays bounded."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import scan_oracle as so
+from paper_2411_17887_b200 import binding as B
+from paper_2411_17887_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+PIECE = 1 << 24
+
+
+@pytest.fixture(scope="module")
+def runner():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from tests.gpu_util import Runner
+    return Runner(4096, 1 << 28)
+
+
+def compare_piecewise(got: np.ndarray, x: np.ndarray, dtype: str, exclusive: bool):
+    """1-D arrays: oracle on pieces of 2^24 elements with the running carry passed along."""
+    carry, acarry = 0, 0.0
+    worst = 0.0
+    for lo in range(0, x.size, PIECE):
+        xs = x[lo:lo + PIECE]
+        g = got[lo:lo + PIECE]
+        if dtype == "i8":
+            y = so.scan_i8(xs, exclusive, init=carry)
+            carry = int(y[-1]) + (int(xs[-1]) if exclusive else 0)
+            assert np.array_equal(g, so.wrap_int32(y)), f"mismatch in piece at {lo}"
+        else:
+            x64 = so.widen(xs, dtype)
+            y, a = so.scan_f64(x64, exclusive, init=carry)
+            a = a + acarry
+            carry = float(y[-1]) + (float(x64[-1]) if exclusive else 0.0)
+            acarry = float(a[-1]) + (abs(float(x64[-1])) if exclusive else 0.0)
+            err = np.abs(g.astype(np.float64) - y)
+            tol = so.float_tolerance(a)
+            assert (err <= tol).all(), f"out of tolerance in piece at {lo}: worst ratio {(err / tol).max()}"
+            worst = max(worst, float((err / tol).max()))
+    return worst
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3", "C5", "C3h"])
+def test_single_array_configs(runner, name):
+    cfg = inputs.CONFIGS[name]
+    x = inputs.make(cfg)
+    from tests.gpu_util import to_device
+    d_in = to_device(x, cfg.dtype)
+    for s in cfg.s:
+        for exclusive in cfg.exclusive:
+            got = runner.run(x, cfg.dtype, s, exclusive, d_in=d_in)
+            compare_piecewise(got, x, cfg.dtype, exclusive)
+            if cfg.dtype == "i8":                      # integer results are identical from run to run
+                again = runner.run(x, cfg.dtype, s, exclusive, d_in=d_in)
+                assert np.array_equal(got, again)
+            st = B.tcu_scan_last_stats()
+            assert st["sxs_products"] == x.size // (s * s)        # the n / s^2 level-0 products
+            assert st["levels_used"] <= max(st["depth_bound"], 5)
+
+
+def test_batched_config_C4(runner):
+    cfg = inputs.CONFIGS["C4"]
+    x = inputs.make(cfg)
+    got = runner.run(x, cfg.dtype, 16, False)
+    block = 256
+    for r0 in range(0, x.shape[0], block):
+        xs = x[r0:r0 + block]
+        y, a = so.scan_f64(so.widen(xs, cfg.dtype))
+        err = np.abs(got[r0:r0 + block].astype(np.float64) - y)
+        assert (err <= so.float_tolerance(a)).all(), f"rows {r0}.."

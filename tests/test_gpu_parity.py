@@ -1,0 +1,137 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Integers must match bit for bit; fp32 outputs must satisfy
+|y - y_ref| <= 1e-5 * sum_{j<=i}|x_j| + 1e-6 with y_ref the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import scan_oracle as so
+from oracle import tcu_model as tm
+from paper_2411_17887_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TILE = 128 * 128
+
+
+@pytest.fixture(scope="module")
+def runner():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from tests.gpu_util import Runner
+    return Runner(64, 1 << 22)
+
+
+def gen(dtype, shape, seed):
+    if dtype == "i8":
+        return inputs.int8_uniform(shape, -127, 127, seed)
+    if dtype == "f16":
+        return inputs.f16_uniform(shape, -1.0, 1.0, seed)
+    return inputs.bf16_normal(shape, seed)
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f16", "bf16"])
+@pytest.mark.parametrize("s", [16, 64, 128])
+def test_level0_is_upsweep_round_0(runner, dtype, s):
+    # After up-sweep round t = 0 of Algorithm 1 every chunk of s elements holds its own scan:
+    # compare with the model's BatchMatMul(x, L_s) on three tiles.
+    n = 3 * TILE
+    x = gen(dtype, n, 40 + s)
+    got = runner.run(x, dtype, s, level0=True)
+    if dtype == "i8":
+        want = tm.batch_matmul(x.astype(np.int64), tm.L_matrix(s))
+        assert np.array_equal(got.astype(np.int64), want)
+    else:
+        x64 = so.widen(x, dtype)
+        want = tm.batch_matmul(x64, tm.L_matrix(s, np.float64))
+        bound = 1e-5 * tm.batch_matmul(np.abs(x64), tm.L_matrix(s, np.float64)) + 1e-6
+        assert (np.abs(got - want) <= bound).all()
+
+
+EDGE_SIZES = [1, 2, 15, 16, 17, 127, 128, 129, 255, 256, 257, 16 * 16 + 1, TILE - 1, TILE, TILE + 1,
+              TILE + 128, 3 * TILE + 5, 5 * TILE - 128]
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f16", "bf16"])
+@pytest.mark.parametrize("exclusive", [False, True])
+def test_edge_sizes(runner, dtype, exclusive):
+    from tests.gpu_util import check
+    for s in (16, 64, 128):
+        for n in EDGE_SIZES:
+            x = gen(dtype, n, 1000 + n % 977 + s)
+            check(runner, x, dtype, s, exclusive)
+
+
+@pytest.mark.parametrize("dtype,s", [("i8", 16), ("i8", 128), ("f16", 16), ("bf16", 64)])
+def test_around_one_wave_of_tiles(runner, dtype, s):
+    # one tile per SM, one less, one more, and a ragged tail: exercises the persistent schedule
+    from tests.gpu_util import check
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for n in (sms * TILE - 1, sms * TILE, sms * TILE + 1, (sms + 1) * TILE + 77, (2 * sms + 3) * TILE + 128 * 9 + 3):
+        for exclusive in (False, True):
+            check(runner, gen(dtype, n, n % 1013), dtype, s, exclusive)
+
+
+def test_all_ones_fp16_is_exact(runner):
+    # every partial sum is an integer <= 2^22, exactly representable in fp32 whatever the association:
+    # a layout or carry bug that the tolerance would hide shows up here
+    n = 1 << 22
+    x = np.ones(n, np.float16)
+    for s in (16, 64, 128):
+        got = runner.run(x, "f16", s)
+        assert np.array_equal(got, np.arange(1, n + 1, dtype=np.float32))
+        got = runner.run(x, "f16", s, exclusive=True)
+        assert np.array_equal(got, np.arange(0, n, dtype=np.float32))
+
+
+def test_int_position_sensitivity(runner):
+    # distinct weights per position: a permuted row / chunk inside a tile cannot cancel out
+    n = 4 * TILE + 128 * 3
+    x = ((np.arange(n) * 37 + (np.arange(n) // 128) * 11) % 251 - 125).astype(np.int8)
+    from tests.gpu_util import check
+    for s in (16, 64, 128):
+        check(runner, x, "i8", s)
+        check(runner, x, "i8", s, True)
+
+
+def test_int_wraps_modulo_2_32(runner):
+    n = 1 << 22
+    x = np.full(n, 127, np.int8)
+    x[: 1 << 21] = 127
+    big = np.concatenate([x] * 1)
+    from tests.gpu_util import check
+    got = check(runner, big, "i8", 16)
+    assert int(got[-1]) == 127 * n                       # no wrap yet at this size ...
+    xx = np.full(1 << 22, -128, np.int8)                 # ... and the most negative input value
+    check(runner, xx, "i8", 16)
+
+
+@pytest.mark.parametrize("dtype", ["i8", "bf16", "f16"])
+def test_batched_rows(runner, dtype):
+    from tests.gpu_util import check
+    for rows, cols in [(1, 128), (3, 128), (5, TILE), (4, 2 * TILE + 128 * 5), (64, 65536), (7, 128 * 129)]:
+        for s in (16, 128):
+            check(runner, gen(dtype, (rows, cols), rows * 7 + cols % 101), dtype, s, False)
+        check(runner, gen(dtype, (rows, cols), rows * 7 + cols % 103), dtype, 64, True)
+
+
+def test_repeatable_and_workspace_reuse(runner):
+    # the same workspace serves different shapes back to back; integer results never change between runs
+    from tests.gpu_util import check
+    x = gen("i8", 200 * TILE + 9, 5)
+    a = check(runner, x, "i8", 16)
+    y = gen("f16", 3 * TILE, 6)
+    check(runner, y, "f16", 64)
+    b = check(runner, x, "i8", 16)
+    assert np.array_equal(a, b)
+
+
+def test_stats_report(runner):
+    from paper_2411_17887_b200 import binding as B
+    n = 1 << 20
+    runner.run(gen("f16", n, 3), "f16", 64)
+    st = B.tcu_scan_last_stats()
+    assert st["tiles"] == n // TILE and st["s"] == 64 and st["sxs_products"] == n // (64 * 64)
+    assert st["depth_bound"] == 2 * 3 and st["levels_used"] == 5 and st["variant"] == 0 and st["upper_level_path"] == 0
+    assert st["mma_instructions"] == st["tiles"] * 2 * 4
