@@ -4,13 +4,13 @@
 //   warp 0    TMA producer: cp.async.bulk.tensor loads of the tile into a shared-memory ring
 //   warp 1    MMA issuer:   tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into TMEM
 //             (Algorithm 1, up-sweep round t = 0: every length-s chunk becomes its local scan)
-//   warp 2    carry scan across tiles: decoupled look-back over per-tile records in global
+//   warps 8-11  totals: read the chunk totals from TMEM, chain them along the row and scan them
+//             across the 128 rows (up-sweep rounds t >= 1), publish the tile total
+//   warps 12-15 carry scan across tiles: decoupled look-back over per-tile records in global
 //             memory (Section 2.2 steps 2-3: totals of the segments, and their scan)
-//   warps 4-7 epilogue: pass 1 reads the chunk totals from TMEM and scans them along the
-//             row and across the 128 rows (up-sweep rounds t >= 1); pass 2 adds chunk, row and
-//             tile carries to every element on the vector ALUs (down-sweep; the paper's
-//             discussion section recommends a vector unit for this add), stages the result
-//             in swizzled shared memory and writes it with TMA stores.
+//   warps 4-7 carry add and store: add chunk, row and tile carries to every element on the
+//             vector ALUs (down-sweep; the paper's discussion section recommends a vector unit
+//             for this add), stage the result in swizzled shared memory, write it with TMA stores
 // Every wait is bounded; a wait that runs out records TCU_ERR_TIMEOUT in the workspace
 // header, and the CTA winds down (drains its copies, frees TMEM) instead of spinning.
 #pragma once
@@ -26,14 +26,16 @@ constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM 
 constexpr int kTileCols = 128;          // elements per tile row
 constexpr int kTileElems = kTileRows * kTileCols;
 constexpr int kNumAcc = 4;              // TMEM accumulators (128 columns each, 512 in all)
-constexpr int kRunAhead = 2;            // tiles by which epilogue pass 1 leads pass 2
 constexpr int kOutChunks = 6;           // ring of 16 KB output staging buffers (32 columns x 128 rows)
 constexpr int kOutChunkBytes = 32 * 4 * kTileRows;
 constexpr int kMaxInStages = 6;
+constexpr int kLookBack = 5;             // records fetched per lane and round of the cross-tile look-back
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kEpilogueThreads = 128;
-constexpr int kFirstEpilogueWarp = 4;
+constexpr int kFirstEpilogueWarp = 4;    // warps 4-7: carry add and store
+constexpr int kFirstTotalsWarp = 8;      // warps 8-11: totals of rows and tile
+constexpr int kFirstLookbackWarp = 12;   // warps 12-15: cross-tile look-back, one warp per accumulator slot
 
 // workspace: 256-byte header, then one 16-byte record per tile
 constexpr int kHeaderBytes = 256;
@@ -315,7 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         for (int i = 0; i < kNumAcc; ++i) {
             mbar_init(smem_u32(&ctl->acc_full[i]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[i]), kEpilogueThreads);
-            mbar_init(smem_u32(&ctl->agg_ready[i]), 1);
+            mbar_init(smem_u32(&ctl->agg_ready[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
         }
         ctl->abort_flag = 0;
@@ -413,54 +415,72 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 mma_commit(smem_u32(&ctl->acc_full[slot]));    // the accumulator is complete
             }
         }
-    } else if (warp == 2) {
+    } else if (warp >= kFirstLookbackWarp) {
         // ------------------------------------------------------------------ cross-tile carry scan
-        for (uint32_t j = 0; j < my_tiles; ++j) {
-            uint32_t t = first_tile + j * stride;
-            uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+        // One warp per accumulator slot, so that the look-backs of the tiles in flight overlap.
+        const uint32_t slot = warp - kFirstLookbackWarp;
+        for (uint32_t j = slot; j < my_tiles; j += kNumAcc) {
+            const uint32_t t = first_tile + j * stride;
+            const uint32_t ua = j / kNumAcc;
             if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[slot]), ua & 1))) break;
             const CarryT agg = CO::dec(ctl->agg_slot[slot]);
             const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
             CarryT prefix = CarryT(0);
-            if (static_cast<int>(t) == t0) {
-                if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(agg));
-            } else {
-                if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusPartial, CO::enc(agg));
+            if (static_cast<int>(t) != t0) {       // (the first tile's record was published by the totals warps)
                 int pos = static_cast<int>(t) - 1;
                 bool gave_up = false;
                 while (true) {
-                    int idx = pos - lane;
-                    bool valid = idx >= t0;
-                    uint64_t flag = 0, val = 0;
-                    if (valid) {
-                        const void *rec = records + size_t(idx) * 16;
-                        ld_record(rec, flag, val);
-                        if (static_cast<uint32_t>(flag >> 2) != epoch) {
+                    // every lane fetches kLookBack records at once (distance d = k * 32 + lane behind
+                    // pos), so that a window of 32 * kLookBack predecessors costs one round trip to L2;
+                    // with one CTA per SM that window reaches back to this CTA's own previous tile
+                    uint64_t flag[kLookBack], val[kLookBack];
+                    bool valid[kLookBack];
+#pragma unroll
+                    for (int k = 0; k < kLookBack; ++k) {
+                        int idx = pos - (k * 32 + lane);
+                        valid[k] = idx >= t0;
+                        flag[k] = 0;
+                        val[k] = 0;
+                        if (valid[k]) ld_record(records + size_t(idx) * 16, flag[k], val[k]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < kLookBack; ++k) {
+                        if (valid[k] && static_cast<uint32_t>(flag[k] >> 2) != epoch) {
+                            const void *rec = records + size_t(pos - (k * 32 + lane)) * 16;
                             long long c0 = clock64();
                             uint32_t spins = 0;
                             while (true) {
-                                ld_record(rec, flag, val);
-                                if (static_cast<uint32_t>(flag >> 2) == epoch) break;
+                                __nanosleep(40);
+                                ld_record(rec, flag[k], val[k]);
+                                if (static_cast<uint32_t>(flag[k] >> 2) == epoch) break;
                                 if ((++spins & 0x3F) == 0 && (ctl->abort_flag || clock64() - c0 > kSpinLimitCycles)) {
                                     gave_up = true;
-                                    flag = kStatusInclusive;   // treat as a chain end so that the walk stops
-                                    val = 0;
+                                    flag[k] = kStatusInclusive;   // treat as a chain end so that the walk stops
+                                    val[k] = 0;
                                     break;
                                 }
                             }
                         }
                     }
-                    bool incl = valid && ((flag & 3) == kStatusInclusive);
-                    unsigned m = __ballot_sync(0xffffffffu, incl);
-                    CarryT v = valid ? CO::dec(val) : CarryT(0);
-                    if (m) {
-                        int first = __ffs(m) - 1;              // nearest predecessor whose record is inclusive
-                        if (lane > first) v = CarryT(0);
-                        prefix += warp_sum(v);
-                        break;
+                    CarryT part = CarryT(0);
+                    bool done = false;
+#pragma unroll
+                    for (int k = 0; k < kLookBack; ++k) {
+                        bool incl = valid[k] && ((flag[k] & 3) == kStatusInclusive);
+                        unsigned m = __ballot_sync(0xffffffffu, incl);
+                        CarryT v = valid[k] ? CO::dec(val[k]) : CarryT(0);
+                        if (!done) {
+                            if (m) {
+                                int first = __ffs(m) - 1;      // nearest predecessor whose record is inclusive
+                                if (lane > first) v = CarryT(0);
+                                done = true;
+                            }
+                            part += v;
+                        }
                     }
-                    prefix += warp_sum(v);
-                    pos -= 32;
+                    prefix += warp_sum(part);
+                    if (done) break;
+                    pos -= 32 * kLookBack;
                     if (pos < t0) break;
                 }
                 if (__any_sync(0xffffffffu, gave_up)) {
@@ -478,8 +498,58 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             __syncwarp();
         }
+    } else if (warp >= kFirstTotalsWarp) {
+        // ------------------------------------------------------------------ totals (up-sweep above the product)
+        // Reads the chunk totals of every row from TMEM, chains them along the row, scans the 128
+        // row totals, and publishes the tile total - as early as the accumulator allows, so that the
+        // cross-tile look-back has the whole life of the accumulator to complete.
+        const int r = threadIdx.x - kFirstTotalsWarp * 32;          // tile row owned by this thread = TMEM lane
+        const int wq = r >> 5;
+        const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
+        for (uint32_t j = 0; j < my_tiles; ++j) {
+            const uint32_t t = first_tile + j * stride;
+            const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+            // a wait that ran out is voted on at the barrier below, so that all 128 threads leave together
+            const bool ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
+            tc_fence_after();
+            uint32_t tot[kChunksPerRow];
+#pragma unroll
+            for (int g = 0; g < kChunksPerRow; ++g) tot[g] = tmem_ld1(lane_base + slot * kTileCols + g * S + (S - 1));
+            tmem_ld_wait();
+            uint32_t rowtot = tot[0];
+#pragma unroll
+            for (int g = 1; g < kChunksPerRow; ++g) rowtot = add32<IS_INT>(rowtot, tot[g]);
+            uint32_t inc = rowtot;                                    // inclusive scan across the warp's 32 rows
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t up = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc = add32<IS_INT>(inc, up);
+            }
+            uint32_t exc = __shfl_up_sync(0xffffffffu, inc, 1);
+            if (lane == 0) exc = 0;
+            const int pb = j & 1;
+            if (lane == 31) ctl->warp_tot[pb][wq] = inc;
+            if (named_barrier_or(2, kEpilogueThreads, !ok)) break;
+            uint32_t w0 = ctl->warp_tot[pb][0], w1 = ctl->warp_tot[pb][1], w2 = ctl->warp_tot[pb][2], w3 = ctl->warp_tot[pb][3];
+            uint32_t before = 0;                                      // rows of the earlier warps
+            if (wq >= 1) before = w0;
+            if (wq >= 2) before = add32<IS_INT>(before, w1);
+            if (wq >= 3) before = add32<IS_INT>(before, w2);
+            rowpref[slot * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
+            if (r == 0) {
+                uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
+                CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
+                // the first tile of a scan has nothing before it: its total is already inclusive
+                const uint32_t status = (t % p.tiles_per_row == 0) ? kStatusInclusive : kStatusPartial;
+                st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(a));
+                ctl->agg_slot[slot] = CO::enc(a);
+            }
+            // every thread arrives (release) after its own rowpref entry is written: the look-back warp,
+            // and through it the store warps, then see all 128 entries
+            mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
+        }
     } else if (warp >= kFirstEpilogueWarp) {
-        // ------------------------------------------------------------------ epilogue
+        // ------------------------------------------------------------------ carry add and store (down-sweep)
         const int r = threadIdx.x - kFirstEpilogueWarp * 32;        // tile row owned by this thread = TMEM lane
         const int wq = r >> 5;
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
@@ -487,99 +557,58 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const bool issuer = (r == 0);
         uint32_t chunk_counter = 0;
         bool dead = false;
-
-        for (uint32_t i = 0; i < my_tiles + kRunAhead && !dead; ++i) {
-            if (i < my_tiles) {
-                // ---- pass 1: totals of the row, scan over the 128 rows, tile total
-                const uint32_t j = i;
-                const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
-                // a wait that ran out is voted on at the next barrier, so that all 128 threads leave together
-                const bool ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
-                tc_fence_after();
-                uint32_t tot[kChunksPerRow];
-#pragma unroll
-                for (int g = 0; g < kChunksPerRow; ++g) tot[g] = tmem_ld1(lane_base + slot * kTileCols + g * S + (S - 1));
-                tmem_ld_wait();
-                uint32_t rowtot = tot[0];
-#pragma unroll
-                for (int g = 1; g < kChunksPerRow; ++g) rowtot = add32<IS_INT>(rowtot, tot[g]);
-                uint32_t inc = rowtot;                                // inclusive scan across the warp's 32 rows
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t up = __shfl_up_sync(0xffffffffu, inc, o);
-                    if (lane >= o) inc = add32<IS_INT>(inc, up);
-                }
-                uint32_t exc = __shfl_up_sync(0xffffffffu, inc, 1);
-                if (lane == 0) exc = 0;
-                const int pb = j & 1;
-                if (lane == 31) ctl->warp_tot[pb][wq] = inc;
-                if (named_barrier_or(1, kEpilogueThreads, !ok)) { dead = true; break; }
-                uint32_t w0 = ctl->warp_tot[pb][0], w1 = ctl->warp_tot[pb][1], w2 = ctl->warp_tot[pb][2], w3 = ctl->warp_tot[pb][3];
-                uint32_t before = 0;                                  // rows of the earlier warps
-                if (wq >= 1) before = w0;
-                if (wq >= 2) before = add32<IS_INT>(before, w1);
-                if (wq >= 3) before = add32<IS_INT>(before, w2);
-                rowpref[slot * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
-                if (issuer) {
-                    uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
-                    CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
-                    ctl->agg_slot[slot] = CO::enc(a);
-                    mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
-                }
+        for (uint32_t j = 0; j < my_tiles && !dead; ++j) {
+            const uint32_t t = first_tile + j * stride;
+            const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+            bool ok = w.wait(smem_u32(&ctl->carry_ready[slot]), ua & 1);
+            ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1) && ok;   // (already complete: the totals came from it)
+            tc_fence_after();
+            const int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
+            uint32_t base;                                            // sum of everything before this row
+            {
+                CarryT carry = CO::dec(ctl->carry_slot[slot]);
+                uint32_t rp = rowpref[slot * kTileRows + r];
+                if (IS_INT) base = uint32_t(carry) + rp;
+                else base = __float_as_uint(static_cast<float>(double(carry) + double(__uint_as_float(rp))));
             }
-            if (i >= kRunAhead) {
-                // ---- pass 2: add the carries, stage, store
-                const uint32_t j = i - kRunAhead;
-                const uint32_t t = first_tile + j * stride;
-                const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
-                const bool ok = w.wait(smem_u32(&ctl->carry_ready[slot]), ua & 1);
-                const int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
-                uint32_t base;                                        // sum of everything before this row
-                {
-                    CarryT carry = CO::dec(ctl->carry_slot[slot]);
-                    uint32_t rp = rowpref[slot * kTileRows + r];
-                    if (IS_INT) base = uint32_t(carry) + rp;
-                    else base = __float_as_uint(static_cast<float>(double(carry) + double(__uint_as_float(rp))));
-                }
-                const bool level0 = p.level0_only != 0;
-                if (level0) base = 0;
-                uint32_t run = base;                                  // sum of everything before the current chunk
-                uint32_t prev = base;                                 // value of the element to the left (exclusive form)
+            const bool level0 = p.level0_only != 0;
+            if (level0) base = 0;
+            uint32_t run = base;                                      // sum of everything before the current chunk
+            uint32_t prev = base;                                     // value of the element to the left (exclusive form)
 #pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t d[32];
-                    tmem_ld32(lane_base + slot * kTileCols + q * 32, d);
-                    tmem_ld_wait();
-                    uint32_t o[32];
+            for (int q = 0; q < 4; ++q) {
+                uint32_t d[32];
+                tmem_ld32(lane_base + slot * kTileCols + q * 32, d);
+                tmem_ld_wait();
+                uint32_t o[32];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        uint32_t v = add32<IS_INT>(d[c], run);
-                        o[c] = EXCL ? prev : v;
-                        prev = v;
-                        const bool chunk_end = (S <= 32) ? (((c + 1) % S) == 0) : (c == 31 && (((q + 1) * 32) % S) == 0);
-                        if (chunk_end && !level0) run = v;            // end of a chunk: its total joins the carry
-                    }
-                    if (level0 && EXCL) {                             // not a meaningful combination; keep it defined
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) o[c] = d[c];
-                    }
-                    const uint32_t buf = out_base + (chunk_counter % kOutChunks) * kOutChunkBytes + r * 128;
-#pragma unroll
-                    for (int c4 = 0; c4 < 8; ++c4)
-                        st_shared_v4(buf + ((c4 ^ (r & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
-                    fence_proxy_async_smem();
-                    if (issuer) bulk_wait_read<kOutChunks - 2>();      // the buffer of the next chunk has been drained
-                    if (named_barrier_or(1, kEpilogueThreads, !ok)) { dead = true; break; }
-                    if (issuer) {
-                        tma_store_3d(&p.tmap_out, out_base + (chunk_counter % kOutChunks) * kOutChunkBytes, q * 32, lt * kTileRows, scan_row);
-                        bulk_commit();
-                    }
-                    ++chunk_counter;
+                for (int c = 0; c < 32; ++c) {
+                    uint32_t v = add32<IS_INT>(d[c], run);
+                    o[c] = EXCL ? prev : v;
+                    prev = v;
+                    const bool chunk_end = (S <= 32) ? (((c + 1) % S) == 0) : (c == 31 && (((q + 1) * 32) % S) == 0);
+                    if (chunk_end && !level0) run = v;                // end of a chunk: its total joins the carry
                 }
-                if (dead) break;
-                tc_fence_before();
-                mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
+                if (level0 && EXCL) {                                 // not a meaningful combination; keep it defined
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) o[c] = d[c];
+                }
+                const uint32_t buf = out_base + (chunk_counter % kOutChunks) * kOutChunkBytes + r * 128;
+#pragma unroll
+                for (int c4 = 0; c4 < 8; ++c4)
+                    st_shared_v4(buf + ((c4 ^ (r & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
+                fence_proxy_async_smem();
+                if (issuer) bulk_wait_read<kOutChunks - 2>();          // the buffer of the next chunk has been drained
+                if (named_barrier_or(1, kEpilogueThreads, !ok)) { dead = true; break; }
+                if (issuer) {
+                    tma_store_3d(&p.tmap_out, out_base + (chunk_counter % kOutChunks) * kOutChunkBytes, q * 32, lt * kTileRows, scan_row);
+                    bulk_commit();
+                }
+                ++chunk_counter;
             }
+            if (dead) break;
+            tc_fence_before();
+            mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
         }
         if (issuer) bulk_wait_all();
     }
