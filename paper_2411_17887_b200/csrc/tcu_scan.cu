@@ -128,7 +128,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     const int b_atoms = (seff * eb + 127) / 128;
     const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
     const uint32_t stage_bytes = kTileElems * eb;
-    const size_t fixed = kConstOffset + b_bytes + size_t(kOutChunks) * kOutChunkBytes + 1024;  // + alignment slack
+    const size_t fixed = kConstOffset + b_bytes + size_t(kOutRingBytes) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kMaxInStages) in_stages = kMaxInStages;
     if (in_stages > 4 && eb == 2) in_stages = 4;
@@ -180,7 +180,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         }
         {
             const cuuint64_t strides[2] = {cuuint64_t(kTileCols) * 4, pitch_elems * 4};
-            const cuuint32_t box[3] = {32, cuuint32_t(kTileRows), 1};
+            const cuuint32_t box[3] = {32, 32, 1};   // one slab: 32 columns x 32 rows, stored by one warp
             CUtensorMapDataType ty = dt == TCU_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
             CUresult r = encode(&prm.tmap_out, ty, 3, d_out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,

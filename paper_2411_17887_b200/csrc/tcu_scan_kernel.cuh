@@ -1,16 +1,17 @@
 // Single-pass tensor-core-unit scan for sm_100a: device code.
 //
-// One persistent CTA per SM walks 128 x 128-element tiles in increasing order.
+// One persistent CTA per SM claims 128 x 128-element tiles in increasing order from a ticket counter.
 //   warp 0    TMA producer: cp.async.bulk.tensor loads of the tile into a shared-memory ring
 //   warp 1    MMA issuer:   tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into TMEM
 //             (Algorithm 1, up-sweep round t = 0: every length-s chunk becomes its local scan)
-//   warps 8-11  totals: read the chunk totals from TMEM, chain them along the row and scan them
+//   warps 12-15 totals: read the chunk totals from TMEM, chain them along the row and scan them
 //             across the 128 rows (up-sweep rounds t >= 1), publish the tile total
-//   warps 12-15 carry scan across tiles: decoupled look-back over per-tile records in global
+//   warps 16-19 carry scan across tiles: decoupled look-back over per-tile records in global
 //             memory (Section 2.2 steps 2-3: totals of the segments, and their scan)
-//   warps 4-7 carry add and store: add chunk, row and tile carries to every element on the
-//             vector ALUs (down-sweep; the paper's discussion section recommends a vector unit
-//             for this add), stage the result in swizzled shared memory, write it with TMA stores
+//   warps 4-11  carry add and store (two groups of four warps taking alternate tiles): add chunk,
+//             row and tile carries to every element on the vector ALUs (down-sweep; the paper's
+//             discussion section recommends a vector unit for this add), stage the result in
+//             swizzled shared memory, write it with TMA stores
 // Every wait is bounded; a wait that runs out records TCU_ERR_TIMEOUT in the workspace
 // header, and the CTA winds down (drains its copies, frees TMEM) instead of spinning.
 #pragma once
@@ -26,16 +27,29 @@ constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM 
 constexpr int kTileCols = 128;          // elements per tile row
 constexpr int kTileElems = kTileRows * kTileCols;
 constexpr int kNumAcc = 4;              // TMEM accumulators (128 columns each, 512 in all)
-constexpr int kOutChunks = 6;           // ring of 16 KB output staging buffers (32 columns x 128 rows)
-constexpr int kOutChunkBytes = 32 * 4 * kTileRows;
+#ifndef TCU_STORE_GROUPS
+#define TCU_STORE_GROUPS 2
+#endif
+#ifndef TCU_LOOKBACK
+#define TCU_LOOKBACK 1
+#endif
+#ifndef TCU_STATIC_TILES
+#define TCU_STATIC_TILES 1
+#endif
+constexpr int kStoreGroups = TCU_STORE_GROUPS;         // groups of 4 store warps; group g handles the tiles with j % kStoreGroups == g
+constexpr int kSlabBytes = 32 * 4 * 32; // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
+constexpr int kSlabsPerWarp = 6 / kStoreGroups;        // ring depth of every store warp
+constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabsPerWarp * kSlabBytes;
+constexpr int kTileRing = 16;           // ring of claimed tile numbers handed from the producer to the MMA warp
+constexpr uint32_t kNoTile = 0xFFFFFFFFu;   // "no more tiles" marker pushed through the pipeline
 constexpr int kMaxInStages = 6;
-constexpr int kLookBack = 5;             // records fetched per lane and round of the cross-tile look-back
+constexpr int kLookBack = TCU_LOOKBACK;             // records fetched per lane and round of the cross-tile look-back
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
-constexpr int kThreads = 512;
 constexpr int kEpilogueThreads = 128;
-constexpr int kFirstEpilogueWarp = 4;    // warps 4-7: carry add and store
-constexpr int kFirstTotalsWarp = 8;      // warps 8-11: totals of rows and tile
-constexpr int kFirstLookbackWarp = 12;   // warps 12-15: cross-tile look-back, one warp per accumulator slot
+constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
+constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
+constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back: one warp per accumulator slot
+constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumAcc);
 
 // workspace: 256-byte header, then one 16-byte record per tile
 constexpr int kHeaderBytes = 256;
@@ -45,7 +59,8 @@ struct WsHeader {
     uint32_t epoch;      // launches completed on this workspace
     uint32_t done;       // CTAs of the running launch that have finished
     uint32_t error;      // tcu_status_t recorded by a bounded wait that ran out
-    uint32_t pad[61];
+    uint32_t ticket;     // next tile number to hand out (tiles are claimed in increasing order)
+    uint32_t pad[60];
 };
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
 
@@ -74,6 +89,8 @@ struct SmemCtl {
     uint64_t agg_slot[kNumAcc];      // tile total (bits of a double, or a zero-extended uint32)
     uint64_t carry_slot[kNumAcc];    // sum of all earlier tiles of the same scan
     uint32_t warp_tot[2][4];         // cross-warp hop of the 128-row scan (double buffered)
+    uint32_t tile_of[kTileRing];     // tile number of the j-th tile claimed by this CTA (producer -> MMA warp)
+    uint32_t slot_tile[kNumAcc];     // tile number held by each accumulator slot (MMA warp -> everyone after it)
     uint32_t tmem_base;
     uint32_t epoch;
     volatile uint32_t abort_flag;
@@ -315,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             mbar_init(smem_u32(&ctl->empty[i]), 1);
         }
         for (int i = 0; i < kNumAcc; ++i) {
-            mbar_init(smem_u32(&ctl->acc_full[i]), 1);
+            mbar_init(smem_u32(&ctl->acc_full[i]), 2);
             mbar_init(smem_u32(&ctl->acc_empty[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->agg_ready[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
@@ -356,19 +373,27 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     const uint32_t epoch = ctl->epoch;
     Waiter w{ctl, hdr};
 
-    const uint32_t first_tile = blockIdx.x;
-    const uint32_t stride = gridDim.x;
-    const uint32_t my_tiles = (p.tiles_total > first_tile) ? (p.tiles_total - first_tile + stride - 1) / stride : 0;
-
+    // Tiles are claimed at run time, in increasing order, from a ticket counter in the workspace:
+    // whoever holds tile t knows that every tile before t is held by a CTA that is already running,
+    // so the look-back below always makes progress, and a slow SM simply claims fewer tiles.  When
+    // the tickets run out the producer pushes kNumAcc "no more tiles" markers through the pipeline,
+    // one per accumulator slot, so that every role (and every per-slot look-back warp) sees one.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t issued = 0;
-            for (uint32_t j = 0; j < my_tiles; ++j) {
-                uint32_t t = first_tile + j * stride;
+            uint32_t issued = 0, markers = 0;
+            for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
+                uint32_t t = (markers == 0) ? (TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u)) : kNoTile;
+                if (t >= p.tiles_total) t = kNoTile;
+                ctl->tile_of[j % kTileRing] = t;
                 uint32_t bar = smem_u32(&ctl->full[stage]);
+                if (t == kNoTile) {
+                    mbar_arrive(bar);
+                    if (++markers == kNumAcc) break;
+                    continue;
+                }
                 mbar_expect_tx(bar, kStageBytes);
                 int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
 #pragma unroll
@@ -393,11 +418,21 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         if (lane == 0) {
             const uint32_t idesc = make_idesc(p.dtype, kSeff);
             const uint32_t b_base = smem_u32(const_region);
-            for (uint32_t j = 0; j < my_tiles; ++j) {
+            uint32_t markers = 0;
+            for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
                 uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
                 if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                const uint32_t t = ctl->tile_of[j % kTileRing];
                 if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
+                ctl->slot_tile[slot] = t;
+                if (t == kNoTile) {
+                    mbar_arrive(smem_u32(&ctl->empty[stage]));
+                    mbar_arrive(smem_u32(&ctl->acc_full[slot]));
+                    mbar_arrive(smem_u32(&ctl->acc_full[slot]));
+                    if (++markers == kNumAcc) break;
+                    continue;
+                }
                 tc_fence_after();
                 const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
 #pragma unroll
@@ -412,17 +447,21 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     }
                 }
                 mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once the MMAs have read it
-                mma_commit(smem_u32(&ctl->acc_full[slot]));    // the accumulator is complete
+                mma_commit(smem_u32(&ctl->acc_full[slot]));    // first arrival: the accumulator is complete
+                mbar_arrive(smem_u32(&ctl->acc_full[slot]));   // second arrival (release): slot_tile[slot] is written
             }
         }
     } else if (warp >= kFirstLookbackWarp) {
         // ------------------------------------------------------------------ cross-tile carry scan
         // One warp per accumulator slot, so that the look-backs of the tiles in flight overlap.
         const uint32_t slot = warp - kFirstLookbackWarp;
-        for (uint32_t j = slot; j < my_tiles; j += kNumAcc) {
-            const uint32_t t = first_tile + j * stride;
-            const uint32_t ua = j / kNumAcc;
+        for (uint32_t ua = 0;; ++ua) {
             if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[slot]), ua & 1))) break;
+            const uint32_t t = ctl->slot_tile[slot];
+            if (t == kNoTile) {
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->carry_ready[slot]));
+                break;
+            }
             const CarryT agg = CO::dec(ctl->agg_slot[slot]);
             const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
             CarryT prefix = CarryT(0);
@@ -431,8 +470,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 bool gave_up = false;
                 while (true) {
                     // every lane fetches kLookBack records at once (distance d = k * 32 + lane behind
-                    // pos), so that a window of 32 * kLookBack predecessors costs one round trip to L2;
-                    // with one CTA per SM that window reaches back to this CTA's own previous tile
+                    // pos), so that a window of 32 * kLookBack predecessors costs one round trip to L2
                     uint64_t flag[kLookBack], val[kLookBack];
                     bool valid[kLookBack];
 #pragma unroll
@@ -506,11 +544,18 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const int r = threadIdx.x - kFirstTotalsWarp * 32;          // tile row owned by this thread = TMEM lane
         const int wq = r >> 5;
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
-        for (uint32_t j = 0; j < my_tiles; ++j) {
-            const uint32_t t = first_tile + j * stride;
+        uint32_t markers = 0;
+        for (uint32_t j = 0;; ++j) {
             const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
-            // a wait that ran out is voted on at the barrier below, so that all 128 threads leave together
+            // a wait that ran out is voted on, so that all 128 threads leave together
             const bool ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
+            if (named_barrier_or(2, kEpilogueThreads, !ok)) break;
+            const uint32_t t = ctl->slot_tile[slot];
+            if (t == kNoTile) {
+                mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
+                if (++markers == kNumAcc) break;
+                continue;
+            }
             tc_fence_after();
             uint32_t tot[kChunksPerRow];
 #pragma unroll
@@ -529,7 +574,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (lane == 0) exc = 0;
             const int pb = j & 1;
             if (lane == 31) ctl->warp_tot[pb][wq] = inc;
-            if (named_barrier_or(2, kEpilogueThreads, !ok)) break;
+            named_barrier_sync(2, kEpilogueThreads);
             uint32_t w0 = ctl->warp_tot[pb][0], w1 = ctl->warp_tot[pb][1], w2 = ctl->warp_tot[pb][2], w3 = ctl->warp_tot[pb][3];
             uint32_t before = 0;                                      // rows of the earlier warps
             if (wq >= 1) before = w0;
@@ -548,20 +593,23 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             // and through it the store warps, then see all 128 entries
             mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
         }
-    } else if (warp >= kFirstEpilogueWarp) {
+    } else if (warp >= kFirstStoreWarp) {
         // ------------------------------------------------------------------ carry add and store (down-sweep)
-        const int r = threadIdx.x - kFirstEpilogueWarp * 32;        // tile row owned by this thread = TMEM lane
-        const int wq = r >> 5;
+        // Every warp works alone on its 32 rows: TMEM -> registers -> (add carries) -> its own ring of
+        // swizzled 4 KB slabs -> one TMA store per slab.  No barrier between the warps.
+        const int group = (warp - kFirstStoreWarp) >> 2;
+        const int wq = warp & 3;                                    // TMEM lane quarter this warp may read
+        const int r = wq * 32 + lane;                               // tile row owned by this thread
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
-        const uint32_t out_base = smem_u32(out_ring);
-        const bool issuer = (r == 0);
-        uint32_t chunk_counter = 0;
-        bool dead = false;
-        for (uint32_t j = 0; j < my_tiles && !dead; ++j) {
-            const uint32_t t = first_tile + j * stride;
+        const uint32_t ring = smem_u32(out_ring) + ((warp - kFirstStoreWarp) * kSlabsPerWarp) * kSlabBytes;
+        uint32_t slab_counter = 0;
+        for (uint32_t j = group;; j += kStoreGroups) {
             const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
             bool ok = w.wait(smem_u32(&ctl->carry_ready[slot]), ua & 1);
             ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1) && ok;   // (already complete: the totals came from it)
+            if (!__all_sync(0xffffffffu, ok)) break;
+            const uint32_t t = ctl->slot_tile[slot];
+            if (t == kNoTile) break;
             tc_fence_after();
             const int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
             uint32_t base;                                            // sum of everything before this row
@@ -579,6 +627,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             for (int q = 0; q < 4; ++q) {
                 uint32_t d[32];
                 tmem_ld32(lane_base + slot * kTileCols + q * 32, d);
+                if (lane == 0) bulk_wait_read<kSlabsPerWarp - 1>();    // the slab about to be written has been drained
                 tmem_ld_wait();
                 uint32_t o[32];
 #pragma unroll
@@ -593,24 +642,24 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 #pragma unroll
                     for (int c = 0; c < 32; ++c) o[c] = d[c];
                 }
-                const uint32_t buf = out_base + (chunk_counter % kOutChunks) * kOutChunkBytes + r * 128;
+                __syncwarp();
+                const uint32_t slab = ring + (slab_counter % kSlabsPerWarp) * kSlabBytes;
+                const uint32_t buf = slab + lane * 128;
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4)
-                    st_shared_v4(buf + ((c4 ^ (r & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
+                    st_shared_v4(buf + ((c4 ^ (lane & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
                 fence_proxy_async_smem();
-                if (issuer) bulk_wait_read<kOutChunks - 2>();          // the buffer of the next chunk has been drained
-                if (named_barrier_or(1, kEpilogueThreads, !ok)) { dead = true; break; }
-                if (issuer) {
-                    tma_store_3d(&p.tmap_out, out_base + (chunk_counter % kOutChunks) * kOutChunkBytes, q * 32, lt * kTileRows, scan_row);
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_3d(&p.tmap_out, slab, q * 32, lt * kTileRows + wq * 32, scan_row);
                     bulk_commit();
                 }
-                ++chunk_counter;
+                ++slab_counter;
             }
-            if (dead) break;
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
         }
-        if (issuer) bulk_wait_all();
+        if (lane == 0) bulk_wait_all();
     }
 
     // ---- tear-down
@@ -623,6 +672,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         uint32_t old = atomicAdd(&hdr->done, 1u);
         if (old == gridDim.x - 1) {          // last CTA: the launch is over, open the next epoch
             hdr->done = 0;
+            hdr->ticket = 0;
             __threadfence();
             hdr->epoch = epoch;
         }
