@@ -128,10 +128,9 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     const int b_atoms = (seff * eb + 127) / 128;
     const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
     const uint32_t stage_bytes = kTileElems * eb;
-    const size_t fixed = kConstOffset + b_bytes + size_t(kOutRingBytes) + 1024;  // + alignment slack
+    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kMaxInStages) in_stages = kMaxInStages;
-    if (in_stages > 4 && eb == 2) in_stages = 4;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
     const size_t smem = fixed + size_t(in_stages) * stage_bytes;
 
@@ -145,7 +144,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     st.variant = 0;
     st.upper_level_path = 0;
     st.tiles = tiles;
-    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32));
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32);  // U_s products + row-total products
     st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
     // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
     // scan over the tiles (absent for a single tile), carry add

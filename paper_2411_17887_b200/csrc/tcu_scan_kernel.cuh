@@ -1,17 +1,21 @@
 // Single-pass tensor-core-unit scan for sm_100a: device code.
 //
-// One persistent CTA per SM claims 128 x 128-element tiles in increasing order from a ticket counter.
-//   warp 0    TMA producer: cp.async.bulk.tensor loads of the tile into a shared-memory ring
-//   warp 1    MMA issuer:   tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into TMEM
-//             (Algorithm 1, up-sweep round t = 0: every length-s chunk becomes its local scan)
-//   warps 12-15 totals: read the chunk totals from TMEM, chain them along the row and scan them
-//             across the 128 rows (up-sweep rounds t >= 1), publish the tile total
-//   warps 16-19 carry scan across tiles: decoupled look-back over per-tile records in global
-//             memory (Section 2.2 steps 2-3: totals of the segments, and their scan)
-//   warps 4-11  carry add and store (two groups of four warps taking alternate tiles): add chunk,
-//             row and tile carries to every element on the vector ALUs (down-sweep; the paper's
-//             discussion section recommends a vector unit for this add), stage the result in
-//             swizzled shared memory, write it with TMA stores
+// One persistent CTA per SM processes 128 x 128-element tiles.  Roles (warps):
+//   0      TMA producer: claims the next tile and loads it into a shared-memory ring
+//   1      MMA issuer, local scans: tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into one of
+//          three TMEM accumulators (Algorithm 1, up-sweep round t = 0: every length-s chunk becomes
+//          its own scan)
+//   2      MMA issuer, row totals: tcgen05.mma  R[128 x 16] = X[128 x 128] * ones  into a ring of
+//          eight small TMEM accumulators, issued as soon as the tile has landed - long before a
+//          full accumulator is free - so that the cross-tile carry scan starts early
+//   3      idle
+//   4-11   carry add and store (two groups of four warps taking alternate tiles): add chunk, row
+//          and tile carries to every element on the vector ALUs (down-sweep; the paper's
+//          discussion section recommends a vector unit for this add), stage the result in
+//          swizzled shared memory, write it with TMA stores
+//   12-15  totals: scan the 128 row totals (up-sweep rounds t >= 1), publish the tile total
+//   16-19  carry scan across tiles: decoupled look-back over per-tile records in global memory
+//          (Section 2.2 steps 2-3: totals of the segments, and their scan)
 // Every wait is bounded; a wait that runs out records TCU_ERR_TIMEOUT in the workspace
 // header, and the CTA winds down (drains its copies, frees TMEM) instead of spinning.
 #pragma once
@@ -23,10 +27,6 @@
 
 namespace tcu {
 
-constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM lanes
-constexpr int kTileCols = 128;          // elements per tile row
-constexpr int kTileElems = kTileRows * kTileCols;
-constexpr int kNumAcc = 4;              // TMEM accumulators (128 columns each, 512 in all)
 #ifndef TCU_STORE_GROUPS
 #define TCU_STORE_GROUPS 2
 #endif
@@ -34,22 +34,37 @@ constexpr int kNumAcc = 4;              // TMEM accumulators (128 columns each, 
 #define TCU_LOOKBACK 1
 #endif
 #ifndef TCU_STATIC_TILES
-#define TCU_STATIC_TILES 1
+#define TCU_STATIC_TILES 0
 #endif
-constexpr int kStoreGroups = TCU_STORE_GROUPS;         // groups of 4 store warps; group g handles the tiles with j % kStoreGroups == g
-constexpr int kSlabBytes = 32 * 4 * 32; // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
-constexpr int kSlabsPerWarp = 6 / kStoreGroups;        // ring depth of every store warp
+#ifndef TCU_SLABS
+#define TCU_SLABS 2
+#endif
+
+constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM lanes
+constexpr int kTileCols = 128;          // elements per tile row
+constexpr int kTileElems = kTileRows * kTileCols;
+constexpr int kNumAcc = 3;              // TMEM accumulators of the local scans (128 columns each)
+constexpr int kNumTot = 8;              // TMEM accumulators of the row totals (16 columns each)
+constexpr int kTotCols = 16;
+constexpr int kTotBase = kNumAcc * kTileCols;            // first TMEM column of the totals ring
+static_assert(kTotBase + kNumTot * kTotCols <= 512, "TMEM has 512 columns");
+constexpr int kStoreGroups = TCU_STORE_GROUPS;           // groups of 4 store warps; group g takes the tiles with j % kStoreGroups == g
+constexpr int kSlabBytes = 32 * 4 * 32;                  // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
+constexpr int kSlabsPerWarp = TCU_SLABS;                 // ring depth of every store warp
 constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabsPerWarp * kSlabBytes;
-constexpr int kTileRing = 16;           // ring of claimed tile numbers handed from the producer to the MMA warp
+constexpr int kTileRing = 16;           // ring of claimed tile numbers (must exceed the tiles a CTA has in flight)
 constexpr uint32_t kNoTile = 0xFFFFFFFFu;   // "no more tiles" marker pushed through the pipeline
-constexpr int kMaxInStages = 6;
-constexpr int kLookBack = TCU_LOOKBACK;             // records fetched per lane and round of the cross-tile look-back
+constexpr int kNumMarkers = 4;          // markers pushed: one per look-back warp
+constexpr int kMaxInStages = 8;
+constexpr int kLookBack = TCU_LOOKBACK; // records fetched per lane and round of the cross-tile look-back
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
+constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
 constexpr int kEpilogueThreads = 128;
+constexpr int kNumLookbackWarps = 4;
 constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
-constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back: one warp per accumulator slot
-constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumAcc);
+constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back
+constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps);
 
 // workspace: 256-byte header, then one 16-byte record per tile
 constexpr int kHeaderBytes = 256;
@@ -68,37 +83,38 @@ constexpr long long kSpinLimitCycles = 2000000000LL;   // about one second at B2
 
 struct alignas(64) ScanParams {
     CUtensorMap tmap_in;      // (128, rows128, batch) view of the input, box 128 B x 128 rows
-    CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 128 rows
+    CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 32
     void *ws;
     uint32_t tiles_total;     // all tiles of the launch
     uint32_t tiles_per_row;   // tiles of one scan (carry chain restarts every tiles_per_row tiles)
     uint32_t in_stages;       // depth of the input ring
-    uint32_t b_bytes;         // shared memory reserved for the constant operand
+    uint32_t b_bytes;         // shared memory reserved for the constant operand I (x) U_s
     uint32_t dtype;           // tcu_dtype_t
     uint32_t level0_only;     // debug: stop after the U_s product (no carries)
 };
 
 // shared-memory bookkeeping (lives at the 1024-aligned base of dynamic shared memory)
 struct SmemCtl {
-    uint64_t full[kMaxInStages];     // TMA -> MMA
-    uint64_t empty[kMaxInStages];    // MMA -> TMA
-    uint64_t acc_full[kNumAcc];      // MMA -> epilogue
-    uint64_t acc_empty[kNumAcc];     // epilogue -> MMA
-    uint64_t agg_ready[kNumAcc];     // epilogue pass 1 -> carry warp
-    uint64_t carry_ready[kNumAcc];   // carry warp -> epilogue pass 2
-    uint64_t agg_slot[kNumAcc];      // tile total (bits of a double, or a zero-extended uint32)
-    uint64_t carry_slot[kNumAcc];    // sum of all earlier tiles of the same scan
+    uint64_t full[kMaxInStages];     // TMA -> both MMA issuers
+    uint64_t empty[kMaxInStages];    // both MMA issuers -> TMA
+    uint64_t acc_full[kNumAcc];      // scan MMAs -> store warps
+    uint64_t acc_empty[kNumAcc];     // store warps -> scan MMA issuer
+    uint64_t tot_full[kNumTot];      // row-total MMAs -> totals warps
+    uint64_t tot_empty[kNumTot];     // store warps -> row-total MMA issuer (the whole ring entry is free again)
+    uint64_t agg_ready[kNumTot];     // totals warps -> look-back warp
+    uint64_t carry_ready[kNumTot];   // look-back warp -> store warps
+    uint64_t agg_slot[kNumTot];      // tile total (bits of a double, or a zero-extended uint32)
+    uint64_t carry_slot[kNumTot];    // sum of all earlier tiles of the same scan
     uint32_t warp_tot[2][4];         // cross-warp hop of the 128-row scan (double buffered)
-    uint32_t tile_of[kTileRing];     // tile number of the j-th tile claimed by this CTA (producer -> MMA warp)
-    uint32_t slot_tile[kNumAcc];     // tile number held by each accumulator slot (MMA warp -> everyone after it)
+    uint32_t tile_of[kTileRing];     // tile number of the j-th tile claimed by this CTA
     uint32_t tmem_base;
     uint32_t epoch;
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 1024;
 static_assert(sizeof(SmemCtl) <= kCtlBytes, "control block too large");
-constexpr int kRowPrefBytes = kNumAcc * kTileRows * 4;
-constexpr int kConstOffset = kCtlBytes + kRowPrefBytes;   // 3072: 1024-aligned
+constexpr int kRowPrefBytes = kNumTot * kTileRows * 4;
+constexpr int kConstOffset = kCtlBytes + kRowPrefBytes;   // 5120: 1024-aligned
 static_assert(kConstOffset % 1024 == 0, "operand regions must be 1024-byte aligned");
 
 // ------------------------------------------------------------------------------------ PTX
@@ -306,15 +322,16 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     constexpr int kSeff = (S > kPer32B) ? S : kPer32B;       // side of the block-diagonal constant I (x) U_s
     constexpr int kSegs = kTileCols / kSeff;                 // MMA groups per tile row
     constexpr int kKSteps = kSeff / kPer32B;                 // accumulating MMAs per group
+    constexpr int kRowKSteps = kTileCols / kPer32B;          // accumulating MMAs of the row-total product
     constexpr int kStageBytes = kTileElems * kElemBytes;     // 16 KB (int8) or 32 KB (16-bit)
     constexpr int kInAtoms = kStageBytes / kAtomBytes;
-    constexpr int kChunksPerRow = kTileCols / S;             // length-s chunks in a tile row
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem);
     uint32_t *rowpref = reinterpret_cast<uint32_t *>(smem + kCtlBytes);
-    uint8_t *const_region = smem + kConstOffset;
+    uint8_t *ones_region = smem + kConstOffset;
+    uint8_t *const_region = ones_region + kOnesBytes;
     uint8_t *in_ring = const_region + p.b_bytes;
     uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
 
@@ -329,11 +346,15 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     if (threadIdx.x == 0) {
         for (int i = 0; i < kMaxInStages; ++i) {
             mbar_init(smem_u32(&ctl->full[i]), 1);
-            mbar_init(smem_u32(&ctl->empty[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 2);
         }
         for (int i = 0; i < kNumAcc; ++i) {
-            mbar_init(smem_u32(&ctl->acc_full[i]), 2);
+            mbar_init(smem_u32(&ctl->acc_full[i]), 1);
             mbar_init(smem_u32(&ctl->acc_empty[i]), kEpilogueThreads);
+        }
+        for (int i = 0; i < kNumTot; ++i) {
+            mbar_init(smem_u32(&ctl->tot_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tot_empty[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->agg_ready[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
         }
@@ -345,9 +366,13 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         tmem_alloc(smem_u32(&ctl->tmem_base), 512);
         tmem_relinquish();
     }
-    // constant operand: row n of the K-major storage holds column n of I (x) U_s, i.e. ones at
-    // k <= n inside the same s-block (U_s is L_s transposed: X U_s = (L_s X^T)^T).
+    // Constant operands.  Row n of the K-major storage of I (x) U_s holds column n, i.e. ones at
+    // k <= n inside the same s-block (U_s is L_s transposed: X U_s = (L_s X^T)^T).  The operand of
+    // the row-total product is all ones, so every 32-byte K-slice of it is the same block.
     {
+        const uint32_t one = IS_INT ? 0x01010101u : ((p.dtype == 2) ? 0x3F803F80u : 0x3C003C00u);
+        uint32_t *oz = reinterpret_cast<uint32_t *>(ones_region);
+        for (uint32_t i = threadIdx.x; i < kOnesBytes / 4; i += kThreads) oz[i] = one;
         uint32_t *cz = reinterpret_cast<uint32_t *>(const_region);
         for (uint32_t i = threadIdx.x; i < p.b_bytes / 4; i += kThreads) cz[i] = 0;
         __syncthreads();
@@ -373,11 +398,11 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     const uint32_t epoch = ctl->epoch;
     Waiter w{ctl, hdr};
 
-    // Tiles are claimed at run time, in increasing order, from a ticket counter in the workspace:
-    // whoever holds tile t knows that every tile before t is held by a CTA that is already running,
-    // so the look-back below always makes progress, and a slow SM simply claims fewer tiles.  When
-    // the tickets run out the producer pushes kNumAcc "no more tiles" markers through the pipeline,
-    // one per accumulator slot, so that every role (and every per-slot look-back warp) sees one.
+    // The j-th tile handled by this CTA is number tile_of[j % kTileRing]: either blockIdx.x + j * gridDim.x
+    // (static order) or the next ticket from the workspace (tiles claimed at run time, in increasing order:
+    // whoever holds tile t knows that every tile before t is held by a CTA that is already running).  When
+    // the tiles run out the producer pushes kNumMarkers "no more tiles" markers through the pipeline, so
+    // that every role - and each of the look-back warps - sees one and stops.
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -385,13 +410,14 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
-                uint32_t t = (markers == 0) ? (TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u)) : kNoTile;
+                uint32_t t = kNoTile;
+                if (markers == 0) t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
                 if (t >= p.tiles_total) t = kNoTile;
                 ctl->tile_of[j % kTileRing] = t;
                 uint32_t bar = smem_u32(&ctl->full[stage]);
                 if (t == kNoTile) {
                     mbar_arrive(bar);
-                    if (++markers == kNumAcc) break;
+                    if (++markers == kNumMarkers) break;
                     continue;
                 }
                 mbar_expect_tx(bar, kStageBytes);
@@ -414,7 +440,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ MMA issuer: local scans
         if (lane == 0) {
             const uint32_t idesc = make_idesc(p.dtype, kSeff);
             const uint32_t b_base = smem_u32(const_region);
@@ -423,16 +449,12 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 uint32_t stage = j % num_in, u = j / num_in;
                 uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
                 if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
-                const uint32_t t = ctl->tile_of[j % kTileRing];
-                if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
-                ctl->slot_tile[slot] = t;
-                if (t == kNoTile) {
+                if (ctl->tile_of[j % kTileRing] == kNoTile) {
                     mbar_arrive(smem_u32(&ctl->empty[stage]));
-                    mbar_arrive(smem_u32(&ctl->acc_full[slot]));
-                    mbar_arrive(smem_u32(&ctl->acc_full[slot]));
-                    if (++markers == kNumAcc) break;
+                    if (++markers == kNumMarkers) break;
                     continue;
                 }
+                if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
                 tc_fence_after();
                 const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
 #pragma unroll
@@ -446,31 +468,58 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                         mma_issue<IS_INT>(tmem_base + slot * kTileCols + g * kSeff, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
                     }
                 }
-                mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once the MMAs have read it
-                mma_commit(smem_u32(&ctl->acc_full[slot]));    // first arrival: the accumulator is complete
-                mbar_arrive(smem_u32(&ctl->acc_full[slot]));   // second arrival (release): slot_tile[slot] is written
+                mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once both issuers' MMAs have read it
+                mma_commit(smem_u32(&ctl->acc_full[slot]));
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ MMA issuer: row totals
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(p.dtype, kTotCols);
+            const uint64_t bdesc = make_smem_desc(smem_u32(ones_region));
+            uint32_t markers = 0;
+            for (uint32_t j = 0;; ++j) {
+                uint32_t stage = j % num_in, u = j / num_in;
+                uint32_t ts = j % kNumTot, ut = j / kNumTot;
+                if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                if (!w.wait(smem_u32(&ctl->tot_empty[ts]), (ut & 1) ^ 1)) break;
+                if (ctl->tile_of[j % kTileRing] == kNoTile) {
+                    mbar_arrive(smem_u32(&ctl->empty[stage]));
+                    mbar_arrive(smem_u32(&ctl->tot_full[ts]));
+                    if (++markers == kNumMarkers) break;
+                    continue;
+                }
+                tc_fence_after();
+                const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kRowKSteps; ++kk) {
+                    int a_off = kk * 32;
+                    uint64_t adesc = make_smem_desc(a_base + (a_off >> 7) * kAtomBytes + (a_off & 127));
+                    mma_issue<IS_INT>(tmem_base + kTotBase + ts * kTotCols, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                }
+                mma_commit(smem_u32(&ctl->empty[stage]));
+                mma_commit(smem_u32(&ctl->tot_full[ts]));
             }
         }
     } else if (warp >= kFirstLookbackWarp) {
         // ------------------------------------------------------------------ cross-tile carry scan
-        // One warp per accumulator slot, so that the look-backs of the tiles in flight overlap.
-        const uint32_t slot = warp - kFirstLookbackWarp;
-        for (uint32_t ua = 0;; ++ua) {
-            if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[slot]), ua & 1))) break;
-            const uint32_t t = ctl->slot_tile[slot];
+        // kNumLookbackWarps warps take the tiles in turn, so that the look-backs of the tiles in flight overlap.
+        for (uint32_t j = warp - kFirstLookbackWarp;; j += kNumLookbackWarps) {
+            const uint32_t ts = j % kNumTot, ut = j / kNumTot;
+            if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[ts]), ut & 1))) break;
+            const uint32_t t = ctl->tile_of[j % kTileRing];
             if (t == kNoTile) {
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->carry_ready[slot]));
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->carry_ready[ts]));
                 break;
             }
-            const CarryT agg = CO::dec(ctl->agg_slot[slot]);
+            const CarryT agg = CO::dec(ctl->agg_slot[ts]);
             const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
             CarryT prefix = CarryT(0);
             if (static_cast<int>(t) != t0) {       // (the first tile's record was published by the totals warps)
                 int pos = static_cast<int>(t) - 1;
                 bool gave_up = false;
                 while (true) {
-                    // every lane fetches kLookBack records at once (distance d = k * 32 + lane behind
-                    // pos), so that a window of 32 * kLookBack predecessors costs one round trip to L2
+                    // every lane fetches kLookBack records at once (distance d = k * 32 + lane behind pos)
                     uint64_t flag[kLookBack], val[kLookBack];
                     bool valid[kLookBack];
 #pragma unroll
@@ -531,39 +580,34 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
             }
             if (lane == 0) {
-                ctl->carry_slot[slot] = CO::enc(prefix);
-                mbar_arrive(smem_u32(&ctl->carry_ready[slot]));
+                ctl->carry_slot[ts] = CO::enc(prefix);
+                mbar_arrive(smem_u32(&ctl->carry_ready[ts]));
             }
             __syncwarp();
         }
     } else if (warp >= kFirstTotalsWarp) {
         // ------------------------------------------------------------------ totals (up-sweep above the product)
-        // Reads the chunk totals of every row from TMEM, chains them along the row, scans the 128
-        // row totals, and publishes the tile total - as early as the accumulator allows, so that the
-        // cross-tile look-back has the whole life of the accumulator to complete.
+        // Takes the 128 row totals from the small accumulator, scans them across the rows, and
+        // publishes the tile total - as soon as the tile has landed, so that the cross-tile look-back
+        // has several tile times to complete before the store warps need its result.
         const int r = threadIdx.x - kFirstTotalsWarp * 32;          // tile row owned by this thread = TMEM lane
         const int wq = r >> 5;
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
         uint32_t markers = 0;
         for (uint32_t j = 0;; ++j) {
-            const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+            const uint32_t ts = j % kNumTot, ut = j / kNumTot;
             // a wait that ran out is voted on, so that all 128 threads leave together
-            const bool ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
+            const bool ok = w.wait(smem_u32(&ctl->tot_full[ts]), ut & 1);
             if (named_barrier_or(2, kEpilogueThreads, !ok)) break;
-            const uint32_t t = ctl->slot_tile[slot];
+            const uint32_t t = ctl->tile_of[j % kTileRing];
             if (t == kNoTile) {
-                mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
-                if (++markers == kNumAcc) break;
+                mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
+                if (++markers == kNumMarkers) break;
                 continue;
             }
             tc_fence_after();
-            uint32_t tot[kChunksPerRow];
-#pragma unroll
-            for (int g = 0; g < kChunksPerRow; ++g) tot[g] = tmem_ld1(lane_base + slot * kTileCols + g * S + (S - 1));
+            const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + ts * kTotCols);
             tmem_ld_wait();
-            uint32_t rowtot = tot[0];
-#pragma unroll
-            for (int g = 1; g < kChunksPerRow; ++g) rowtot = add32<IS_INT>(rowtot, tot[g]);
             uint32_t inc = rowtot;                                    // inclusive scan across the warp's 32 rows
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -580,18 +624,18 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (wq >= 1) before = w0;
             if (wq >= 2) before = add32<IS_INT>(before, w1);
             if (wq >= 3) before = add32<IS_INT>(before, w2);
-            rowpref[slot * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
+            rowpref[ts * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
             if (r == 0) {
                 uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
                 CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
                 // the first tile of a scan has nothing before it: its total is already inclusive
                 const uint32_t status = (t % p.tiles_per_row == 0) ? kStatusInclusive : kStatusPartial;
                 st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(a));
-                ctl->agg_slot[slot] = CO::enc(a);
+                ctl->agg_slot[ts] = CO::enc(a);
             }
             // every thread arrives (release) after its own rowpref entry is written: the look-back warp,
             // and through it the store warps, then see all 128 entries
-            mbar_arrive(smem_u32(&ctl->agg_ready[slot]));
+            mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
         }
     } else if (warp >= kFirstStoreWarp) {
         // ------------------------------------------------------------------ carry add and store (down-sweep)
@@ -604,18 +648,20 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const uint32_t ring = smem_u32(out_ring) + ((warp - kFirstStoreWarp) * kSlabsPerWarp) * kSlabBytes;
         uint32_t slab_counter = 0;
         for (uint32_t j = group;; j += kStoreGroups) {
+            const uint32_t ts = j % kNumTot, ut = j / kNumTot;
             const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
-            bool ok = w.wait(smem_u32(&ctl->carry_ready[slot]), ua & 1);
-            ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1) && ok;   // (already complete: the totals came from it)
+            bool ok = w.wait(smem_u32(&ctl->carry_ready[ts]), ut & 1);
             if (!__all_sync(0xffffffffu, ok)) break;
-            const uint32_t t = ctl->slot_tile[slot];
+            const uint32_t t = ctl->tile_of[j % kTileRing];
             if (t == kNoTile) break;
+            ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
+            if (!__all_sync(0xffffffffu, ok)) break;
             tc_fence_after();
             const int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
             uint32_t base;                                            // sum of everything before this row
             {
-                CarryT carry = CO::dec(ctl->carry_slot[slot]);
-                uint32_t rp = rowpref[slot * kTileRows + r];
+                CarryT carry = CO::dec(ctl->carry_slot[ts]);
+                uint32_t rp = rowpref[ts * kTileRows + r];
                 if (IS_INT) base = uint32_t(carry) + rp;
                 else base = __float_as_uint(static_cast<float>(double(carry) + double(__uint_as_float(rp))));
             }
@@ -658,6 +704,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
+            // the ring entry of this tile (row prefixes, carry, row-total accumulator, barriers) may be reused
+            mbar_arrive(smem_u32(&ctl->tot_empty[ts]));
         }
         if (lane == 0) bulk_wait_all();
     }

@@ -134,4 +134,4 @@ def test_stats_report(runner):
     st = B.tcu_scan_last_stats()
     assert st["tiles"] == n // TILE and st["s"] == 64 and st["sxs_products"] == n // (64 * 64)
     assert st["depth_bound"] == 2 * 3 and st["levels_used"] == 5 and st["variant"] == 0 and st["upper_level_path"] == 0
-    assert st["mma_instructions"] == st["tiles"] * 2 * 4
+    assert st["mma_instructions"] == st["tiles"] * (2 * 4 + 8)      # U_64 products + row-total products
