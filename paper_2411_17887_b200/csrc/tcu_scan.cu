@@ -130,7 +130,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     const uint32_t stage_bytes = kTileElems * eb;
     const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
-    if (in_stages > kMaxInStages) in_stages = kMaxInStages;
+    if (in_stages > kUseInStages) in_stages = kUseInStages;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
     const size_t smem = fixed + size_t(in_stages) * stage_bytes;
 
@@ -177,16 +177,10 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
         }
-        {
-            const cuuint64_t strides[2] = {cuuint64_t(kTileCols) * 4, pitch_elems * 4};
-            const cuuint32_t box[3] = {32, 32, 1};   // one slab: 32 columns x 32 rows, stored by one warp
-            CUtensorMapDataType ty = dt == TCU_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-            CUresult r = encode(&prm.tmap_out, ty, 3, d_out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
-        }
         prm.ws = d_ws;
+        prm.out = d_out;
+        prm.scan_pitch = cols;
+        prm.rows128 = uint32_t(rows128);
         prm.tiles_total = uint32_t(tiles);
         prm.tiles_per_row = uint32_t(tiles_per_row);
         prm.in_stages = uint32_t(in_stages);
@@ -286,6 +280,18 @@ tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out) {
     *out = g_stats;
     return TCU_OK;
 }
+
+#ifdef TCU_PROFILE
+// Debug build only: point the kernels at a device buffer of 64 counters per CTA.
+int tcu_scan_debug_set_profile_buffer(void *d_buf) {
+    unsigned long long *p = reinterpret_cast<unsigned long long *>(d_buf);
+    return cudaMemcpyToSymbol(tcu::g_prof, &p, sizeof(p)) == cudaSuccess ? 0 : 4;
+}
+int tcu_scan_debug_set_trace_buffer(void *d_buf) {
+    unsigned long long *p = reinterpret_cast<unsigned long long *>(d_buf);
+    return cudaMemcpyToSymbol(tcu::g_trace, &p, sizeof(p)) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 const char *tcu_status_string(tcu_status_t st) {
     switch (st) {

@@ -31,13 +31,10 @@ namespace tcu {
 #define TCU_STORE_GROUPS 2
 #endif
 #ifndef TCU_LOOKBACK
-#define TCU_LOOKBACK 1
+#define TCU_LOOKBACK 2
 #endif
 #ifndef TCU_STATIC_TILES
 #define TCU_STATIC_TILES 0
-#endif
-#ifndef TCU_SLABS
-#define TCU_SLABS 2
 #endif
 
 constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM lanes
@@ -50,21 +47,30 @@ constexpr int kTotBase = kNumAcc * kTileCols;            // first TMEM column of
 static_assert(kTotBase + kNumTot * kTotCols <= 512, "TMEM has 512 columns");
 constexpr int kStoreGroups = TCU_STORE_GROUPS;           // groups of 4 store warps; group g takes the tiles with j % kStoreGroups == g
 constexpr int kSlabBytes = 32 * 4 * 32;                  // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
-constexpr int kSlabsPerWarp = TCU_SLABS;                 // ring depth of every store warp
-constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabsPerWarp * kSlabBytes;
-constexpr int kTileRing = 16;           // ring of claimed tile numbers (must exceed the tiles a CTA has in flight)
+constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabBytes;   // one transposition slab per store warp
+constexpr int kNumCarry = 16;           // tiles a CTA may have between "row totals known" and "stored": ring of carry entries
+constexpr int kTileRing = 32;           // ring of claimed tile numbers (must exceed the tiles a CTA has in flight)
 constexpr uint32_t kNoTile = 0xFFFFFFFFu;   // "no more tiles" marker pushed through the pipeline
-constexpr int kNumMarkers = 4;          // markers pushed: one per look-back warp
-constexpr int kMaxInStages = 8;
+constexpr int kNumLookbackWarps = 5;
+constexpr int kNumMarkers = kNumLookbackWarps;   // markers pushed: one per look-back warp
+#ifndef TCU_MAX_STAGES
+#define TCU_MAX_STAGES 10
+#endif
+#ifndef TCU_PIPE_STORE
+#define TCU_PIPE_STORE 0
+#endif
+constexpr int kMaxInStages = 12;        // size of the barrier arrays
+constexpr int kUseInStages = TCU_MAX_STAGES;   // stages actually used: a tile is claimed when a stage frees, and claiming
+                                        // earlier than its row-total slot frees (kNumTot - kNumAcc tiles ahead) only
+                                        // makes later tiles of other CTAs wait for it
 constexpr int kLookBack = TCU_LOOKBACK; // records fetched per lane and round of the cross-tile look-back
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
 constexpr int kEpilogueThreads = 128;
-constexpr int kNumLookbackWarps = 4;
 constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back
-constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps);
+constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps - 1);   // warp 3 is the first look-back warp
 
 // workspace: 256-byte header, then one 16-byte record per tile
 constexpr int kHeaderBytes = 256;
@@ -79,12 +85,40 @@ struct WsHeader {
 };
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
 
+#ifdef TCU_PROFILE
+// Debug build only: per-CTA cycle counters of where each role waits (64 counters per CTA).
+__device__ unsigned long long *g_prof = nullptr;
+#define PROF_DECL long long prof_t = 0; unsigned long long prof_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}; (void)prof_t;
+#define PROF_T0() prof_t = clock64()
+#define PROF_ADD(k) do { long long n_ = clock64(); prof_a[k] += (unsigned long long)(n_ - prof_t); prof_t = n_; } while (0)
+#define PROF_INC(k, v) prof_a[k] += (v)
+#define PROF_FLUSH(base, cnt) do { if (g_prof) for (int i_ = 0; i_ < (cnt); ++i_) g_prof[blockIdx.x * 64 + (base) + i_] = prof_a[i_]; } while (0)
+__device__ unsigned long long *g_trace = nullptr;   // 8 time stamps per tile
+__device__ __forceinline__ unsigned long long prof_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define TRACE(tile, k) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = prof_now(); } while (0)
+#define TRACE_V(tile, k, v) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = (v); } while (0)
+#else
+#define TRACE(tile, k)
+#define TRACE_V(tile, k, v)
+#define PROF_DECL
+#define PROF_T0()
+#define PROF_ADD(k)
+#define PROF_INC(k, v)
+#define PROF_FLUSH(base, cnt)
+#endif
+
 constexpr long long kSpinLimitCycles = 2000000000LL;   // about one second at B200 clocks
 
 struct alignas(64) ScanParams {
     CUtensorMap tmap_in;      // (128, rows128, batch) view of the input, box 128 B x 128 rows
-    CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 32
     void *ws;
+    void *out;                // output array (4-byte elements)
+    uint64_t scan_pitch;      // elements between consecutive scans (batched), unused for a single array
+    uint32_t rows128;         // full 128-element rows of one scan
     uint32_t tiles_total;     // all tiles of the launch
     uint32_t tiles_per_row;   // tiles of one scan (carry chain restarts every tiles_per_row tiles)
     uint32_t in_stages;       // depth of the input ring
@@ -100,21 +134,22 @@ struct SmemCtl {
     uint64_t acc_full[kNumAcc];      // scan MMAs -> store warps
     uint64_t acc_empty[kNumAcc];     // store warps -> scan MMA issuer
     uint64_t tot_full[kNumTot];      // row-total MMAs -> totals warps
-    uint64_t tot_empty[kNumTot];     // store warps -> row-total MMA issuer (the whole ring entry is free again)
-    uint64_t agg_ready[kNumTot];     // totals warps -> look-back warp
-    uint64_t carry_ready[kNumTot];   // look-back warp -> store warps
-    uint64_t agg_slot[kNumTot];      // tile total (bits of a double, or a zero-extended uint32)
-    uint64_t carry_slot[kNumTot];    // sum of all earlier tiles of the same scan
+    uint64_t tot_empty[kNumTot];     // totals warps -> row-total MMA issuer (read done)
+    uint64_t ring_free[kNumCarry];   // store warps -> totals warps (the carry ring entry may be reused)
+    uint64_t agg_ready[kNumCarry];   // totals warps -> look-back warp
+    uint64_t carry_ready[kNumCarry]; // look-back warp -> store warps
+    uint64_t agg_slot[kNumCarry];    // tile total (bits of a double, or a zero-extended uint32)
+    uint64_t carry_slot[kNumCarry];  // sum of all earlier tiles of the same scan
     uint32_t warp_tot[2][4];         // cross-warp hop of the 128-row scan (double buffered)
     uint32_t tile_of[kTileRing];     // tile number of the j-th tile claimed by this CTA
     uint32_t tmem_base;
     uint32_t epoch;
     volatile uint32_t abort_flag;
 };
-constexpr int kCtlBytes = 1024;
+constexpr int kCtlBytes = 2048;
 static_assert(sizeof(SmemCtl) <= kCtlBytes, "control block too large");
-constexpr int kRowPrefBytes = kNumTot * kTileRows * 4;
-constexpr int kConstOffset = kCtlBytes + kRowPrefBytes;   // 5120: 1024-aligned
+constexpr int kRowPrefBytes = kNumCarry * kTileRows * 4;
+constexpr int kConstOffset = kCtlBytes + kRowPrefBytes;   // 10240: 1024-aligned
 static_assert(kConstOffset % 1024 == 0, "operand regions must be 1024-byte aligned");
 
 // ------------------------------------------------------------------------------------ PTX
@@ -228,6 +263,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t &a, uint32_t &b, uint32_t &c, uint32_t &d) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void st_global_v4(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ void ld_record(const void *p, uint64_t &flag, uint64_t &val) {
     asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(flag), "=l"(val) : "l"(p) : "memory");
@@ -355,6 +396,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         for (int i = 0; i < kNumTot; ++i) {
             mbar_init(smem_u32(&ctl->tot_full[i]), 1);
             mbar_init(smem_u32(&ctl->tot_empty[i]), kEpilogueThreads);
+        }
+        for (int i = 0; i < kNumCarry; ++i) {
+            mbar_init(smem_u32(&ctl->ring_free[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->agg_ready[i]), kEpilogueThreads);
             mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
         }
@@ -407,12 +451,17 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t issued = 0, markers = 0;
+            PROF_DECL
+            PROF_T0();
             for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
+                PROF_ADD(0);
                 uint32_t t = kNoTile;
                 if (markers == 0) t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
                 if (t >= p.tiles_total) t = kNoTile;
+                PROF_ADD(1);
+                PROF_INC(3, 1);
                 ctl->tile_of[j % kTileRing] = t;
                 uint32_t bar = smem_u32(&ctl->full[stage]);
                 if (t == kNoTile) {
@@ -420,6 +469,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     if (++markers == kNumMarkers) break;
                     continue;
                 }
+                TRACE(t, 0);
                 mbar_expect_tx(bar, kStageBytes);
                 int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
 #pragma unroll
@@ -427,7 +477,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     tma_load_3d(smem_u32(in_ring + stage * kStageBytes + a * kAtomBytes), &p.tmap_in,
                                 a * (128 / kElemBytes), lt * kTileRows, scan_row, bar);
                 issued = j + 1;
+                PROF_ADD(2);
             }
+            PROF_FLUSH(0, 4);
             if (ctl->abort_flag) {
                 // drain: loads already issued must land before the CTA may exit
                 uint32_t lo = issued > num_in ? issued - num_in : 0;
@@ -445,16 +497,20 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             const uint32_t idesc = make_idesc(p.dtype, kSeff);
             const uint32_t b_base = smem_u32(const_region);
             uint32_t markers = 0;
+            PROF_DECL
+            PROF_T0();
             for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
                 uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
                 if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                PROF_ADD(0);
                 if (ctl->tile_of[j % kTileRing] == kNoTile) {
                     mbar_arrive(smem_u32(&ctl->empty[stage]));
                     if (++markers == kNumMarkers) break;
                     continue;
                 }
                 if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
+                PROF_ADD(1);
                 tc_fence_after();
                 const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
 #pragma unroll
@@ -470,7 +526,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 }
                 mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once both issuers' MMAs have read it
                 mma_commit(smem_u32(&ctl->acc_full[slot]));
+                PROF_ADD(2);
             }
+            PROF_FLUSH(4, 3);
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ MMA issuer: row totals
@@ -478,17 +536,23 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             const uint32_t idesc = make_idesc(p.dtype, kTotCols);
             const uint64_t bdesc = make_smem_desc(smem_u32(ones_region));
             uint32_t markers = 0;
+            PROF_DECL
+            PROF_T0();
             for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
                 uint32_t ts = j % kNumTot, ut = j / kNumTot;
                 if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                PROF_ADD(0);
                 if (!w.wait(smem_u32(&ctl->tot_empty[ts]), (ut & 1) ^ 1)) break;
+                PROF_ADD(1);
                 if (ctl->tile_of[j % kTileRing] == kNoTile) {
                     mbar_arrive(smem_u32(&ctl->empty[stage]));
                     mbar_arrive(smem_u32(&ctl->tot_full[ts]));
                     if (++markers == kNumMarkers) break;
                     continue;
                 }
+                TRACE(ctl->tile_of[j % kTileRing], 1);
+                TRACE_V(ctl->tile_of[j % kTileRing], 2, blockIdx.x);
                 tc_fence_after();
                 const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
 #pragma unroll
@@ -499,19 +563,26 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 }
                 mma_commit(smem_u32(&ctl->empty[stage]));
                 mma_commit(smem_u32(&ctl->tot_full[ts]));
+                PROF_ADD(2);
             }
+            PROF_FLUSH(8, 3);
         }
-    } else if (warp >= kFirstLookbackWarp) {
+    } else if (warp == 3 || warp >= kFirstLookbackWarp) {
         // ------------------------------------------------------------------ cross-tile carry scan
         // kNumLookbackWarps warps take the tiles in turn, so that the look-backs of the tiles in flight overlap.
-        for (uint32_t j = warp - kFirstLookbackWarp;; j += kNumLookbackWarps) {
-            const uint32_t ts = j % kNumTot, ut = j / kNumTot;
+        PROF_DECL
+        PROF_T0();
+        const uint32_t lbw = (warp == 3) ? 0u : uint32_t(warp - kFirstLookbackWarp + 1);
+        for (uint32_t j = lbw;; j += kNumLookbackWarps) {
+            const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;
             if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[ts]), ut & 1))) break;
+            PROF_ADD(0);
             const uint32_t t = ctl->tile_of[j % kTileRing];
             if (t == kNoTile) {
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->carry_ready[ts]));
                 break;
             }
+            if (lane == 0) TRACE(t, 4);
             const CarryT agg = CO::dec(ctl->agg_slot[ts]);
             const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
             CarryT prefix = CarryT(0);
@@ -519,53 +590,55 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 int pos = static_cast<int>(t) - 1;
                 bool gave_up = false;
                 while (true) {
-                    // every lane fetches kLookBack records at once (distance d = k * 32 + lane behind pos)
+                    // Every lane fetches kLookBack records at once (distance d = k * 32 + lane behind pos), so
+                    // that a window of 32 * kLookBack predecessors costs one round trip to L2.  The windows
+                    // are then examined nearest first, and only a window that is actually needed is waited
+                    // for: the walk stops at the nearest record that already holds an inclusive sum.
                     uint64_t flag[kLookBack], val[kLookBack];
-                    bool valid[kLookBack];
 #pragma unroll
                     for (int k = 0; k < kLookBack; ++k) {
                         int idx = pos - (k * 32 + lane);
-                        valid[k] = idx >= t0;
                         flag[k] = 0;
                         val[k] = 0;
-                        if (valid[k]) ld_record(records + size_t(idx) * 16, flag[k], val[k]);
-                    }
-#pragma unroll
-                    for (int k = 0; k < kLookBack; ++k) {
-                        if (valid[k] && static_cast<uint32_t>(flag[k] >> 2) != epoch) {
-                            const void *rec = records + size_t(pos - (k * 32 + lane)) * 16;
-                            long long c0 = clock64();
-                            uint32_t spins = 0;
-                            while (true) {
-                                __nanosleep(40);
-                                ld_record(rec, flag[k], val[k]);
-                                if (static_cast<uint32_t>(flag[k] >> 2) == epoch) break;
-                                if ((++spins & 0x3F) == 0 && (ctl->abort_flag || clock64() - c0 > kSpinLimitCycles)) {
-                                    gave_up = true;
-                                    flag[k] = kStatusInclusive;   // treat as a chain end so that the walk stops
-                                    val[k] = 0;
-                                    break;
-                                }
-                            }
-                        }
+                        if (idx >= t0) ld_record(records + size_t(idx) * 16, flag[k], val[k]);
                     }
                     CarryT part = CarryT(0);
                     bool done = false;
 #pragma unroll
                     for (int k = 0; k < kLookBack; ++k) {
-                        bool incl = valid[k] && ((flag[k] & 3) == kStatusInclusive);
-                        unsigned m = __ballot_sync(0xffffffffu, incl);
-                        CarryT v = valid[k] ? CO::dec(val[k]) : CarryT(0);
-                        if (!done) {
+                        if (!done) {                               // warp-uniform
+                            const int idx = pos - (k * 32 + lane);
+                            const bool valid = idx >= t0;
+                            if (valid && static_cast<uint32_t>(flag[k] >> 2) != epoch) {
+                                const void *rec = records + size_t(idx) * 16;
+                                long long c0 = clock64();
+                                uint32_t spins = 0;
+                                while (true) {
+                                    __nanosleep(20);
+                                    ld_record(rec, flag[k], val[k]);
+                                    if (static_cast<uint32_t>(flag[k] >> 2) == epoch) break;
+                                    if ((++spins & 0x3F) == 0 && (ctl->abort_flag || clock64() - c0 > kSpinLimitCycles)) {
+                                        gave_up = true;
+                                        flag[k] = kStatusInclusive;   // treat as a chain end so that the walk stops
+                                        val[k] = 0;
+                                        break;
+                                    }
+                                }
+                            }
+                            const bool incl = valid && ((flag[k] & 3) == kStatusInclusive);
+                            const unsigned m = __ballot_sync(0xffffffffu, incl);
+                            CarryT v = valid ? CO::dec(val[k]) : CarryT(0);
                             if (m) {
-                                int first = __ffs(m) - 1;      // nearest predecessor whose record is inclusive
+                                int first = __ffs(m) - 1;          // nearest predecessor whose record is inclusive
                                 if (lane > first) v = CarryT(0);
                                 done = true;
                             }
                             part += v;
+                            if (pos - (k * 32 + 31) <= t0) done = true;   // the window reached the first tile of the scan
                         }
                     }
                     prefix += warp_sum(part);
+                    PROF_INC(2, 1);
                     if (done) break;
                     pos -= 32 * kLookBack;
                     if (pos < t0) break;
@@ -580,11 +653,15 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
             }
             if (lane == 0) {
+                TRACE(t, 5);
                 ctl->carry_slot[ts] = CO::enc(prefix);
                 mbar_arrive(smem_u32(&ctl->carry_ready[ts]));
             }
             __syncwarp();
+            PROF_ADD(1);
+            PROF_INC(3, 1);
         }
+        if (lane == 0) PROF_FLUSH(12 + 4 * (lbw % 4), 4);
     } else if (warp >= kFirstTotalsWarp) {
         // ------------------------------------------------------------------ totals (up-sweep above the product)
         // Takes the 128 row totals from the small accumulator, scans them across the rows, and
@@ -594,20 +671,28 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const int wq = r >> 5;
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
         uint32_t markers = 0;
+        PROF_DECL
+        PROF_T0();
         for (uint32_t j = 0;; ++j) {
-            const uint32_t ts = j % kNumTot, ut = j / kNumTot;
+            const uint32_t tt = j % kNumTot, utt = j / kNumTot;      // row-total accumulator in TMEM
+            const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;   // carry ring entry
             // a wait that ran out is voted on, so that all 128 threads leave together
-            const bool ok = w.wait(smem_u32(&ctl->tot_full[ts]), ut & 1);
+            bool ok = w.wait(smem_u32(&ctl->tot_full[tt]), utt & 1);
+            ok = w.wait(smem_u32(&ctl->ring_free[ts]), (ut & 1) ^ 1) && ok;
+            PROF_ADD(0);
             if (named_barrier_or(2, kEpilogueThreads, !ok)) break;
             const uint32_t t = ctl->tile_of[j % kTileRing];
             if (t == kNoTile) {
+                mbar_arrive(smem_u32(&ctl->tot_empty[tt]));
                 mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
                 if (++markers == kNumMarkers) break;
                 continue;
             }
             tc_fence_after();
-            const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + ts * kTotCols);
+            const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
             tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&ctl->tot_empty[tt]));                // the small accumulator may be refilled
             uint32_t inc = rowtot;                                    // inclusive scan across the warp's 32 rows
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -631,33 +716,44 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 // the first tile of a scan has nothing before it: its total is already inclusive
                 const uint32_t status = (t % p.tiles_per_row == 0) ? kStatusInclusive : kStatusPartial;
                 st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(a));
+                TRACE(t, 3);
                 ctl->agg_slot[ts] = CO::enc(a);
             }
             // every thread arrives (release) after its own rowpref entry is written: the look-back warp,
             // and through it the store warps, then see all 128 entries
             mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
+            PROF_ADD(1);
         }
+        if (r == 0) PROF_FLUSH(28, 2);
     } else if (warp >= kFirstStoreWarp) {
         // ------------------------------------------------------------------ carry add and store (down-sweep)
-        // Every warp works alone on its 32 rows: TMEM -> registers -> (add carries) -> its own ring of
-        // swizzled 4 KB slabs -> one TMA store per slab.  No barrier between the warps.
+        // Every warp works alone on its 32 rows: TMEM -> registers (one row per lane) -> add carries ->
+        // swizzled 4 KB slab in shared memory -> read back with eight lanes per row -> st.global.v4,
+        // so that every store instruction writes four complete 128-byte lines.  No barrier between warps.
         const int group = (warp - kFirstStoreWarp) >> 2;
         const int wq = warp & 3;                                    // TMEM lane quarter this warp may read
         const int r = wq * 32 + lane;                               // tile row owned by this thread
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
-        const uint32_t ring = smem_u32(out_ring) + ((warp - kFirstStoreWarp) * kSlabsPerWarp) * kSlabBytes;
-        uint32_t slab_counter = 0;
+        const uint32_t slab = smem_u32(out_ring) + (warp - kFirstStoreWarp) * kSlabBytes;
+        const int sub = lane >> 3, piece = lane & 7;                // read-back role: row sub (+4i) of the slab, 16-byte piece
+        uint32_t *const out32 = reinterpret_cast<uint32_t *>(p.out);
+        PROF_DECL
+        PROF_T0();
         for (uint32_t j = group;; j += kStoreGroups) {
-            const uint32_t ts = j % kNumTot, ut = j / kNumTot;
+            const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;
             const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
             bool ok = w.wait(smem_u32(&ctl->carry_ready[ts]), ut & 1);
             if (!__all_sync(0xffffffffu, ok)) break;
+            PROF_ADD(0);
             const uint32_t t = ctl->tile_of[j % kTileRing];
             if (t == kNoTile) break;
             ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
             if (!__all_sync(0xffffffffu, ok)) break;
+            PROF_ADD(1);
+            PROF_INC(5, 1);
+            if (lane == 0 && wq == 0) TRACE(t, 6);
             tc_fence_after();
-            const int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
+            const uint32_t scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
             uint32_t base;                                            // sum of everything before this row
             {
                 CarryT carry = CO::dec(ctl->carry_slot[ts]);
@@ -669,12 +765,15 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (level0) base = 0;
             uint32_t run = base;                                      // sum of everything before the current chunk
             uint32_t prev = base;                                     // value of the element to the left (exclusive form)
-#pragma unroll 1
+            const uint32_t row0 = lt * kTileRows + wq * 32;           // first 128-element row of this warp's part of the tile
+            uint32_t *const gbase = out32 + size_t(scan_row) * p.scan_pitch + size_t(row0) * kTileCols + piece * 4;
+            const int rows_here = int(p.rows128) - int(row0);         // rows of this part that exist (ragged last tile)
+            uint32_t d[32];
+            tmem_ld32(lane_base + slot * kTileCols, d);
+#pragma unroll
             for (int q = 0; q < 4; ++q) {
-                uint32_t d[32];
-                tmem_ld32(lane_base + slot * kTileCols + q * 32, d);
-                if (lane == 0) bulk_wait_read<kSlabsPerWarp - 1>();    // the slab about to be written has been drained
                 tmem_ld_wait();
+                PROF_ADD(2);
                 uint32_t o[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
@@ -688,26 +787,37 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 #pragma unroll
                     for (int c = 0; c < 32; ++c) o[c] = d[c];
                 }
-                __syncwarp();
-                const uint32_t slab = ring + (slab_counter % kSlabsPerWarp) * kSlabBytes;
+                // fetch the next 32 columns while this chunk is transposed and stored
+                if (TCU_PIPE_STORE && q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
+                __syncwarp();                                         // the slab has been read back by every lane
                 const uint32_t buf = slab + lane * 128;
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4)
                     st_shared_v4(buf + ((c4 ^ (lane & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
-                fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) {
-                    tma_store_3d(&p.tmap_out, slab, q * 32, lt * kTileRows + wq * 32, scan_row);
-                    bulk_commit();
+                PROF_ADD(3);
+                uint32_t a[32];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + sub;                       // slab row = tile row row0 + rr
+                    ld_shared_v4(slab + rr * 128 + ((piece ^ (rr & 7)) << 4), a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
                 }
-                ++slab_counter;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + sub;
+                    if (rr < rows_here)
+                        st_global_v4(gbase + size_t(rr) * kTileCols + q * 32, a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+                }
+                PROF_ADD(4);
+                if (!TCU_PIPE_STORE && q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
             }
+            if (lane == 0 && wq == 0) TRACE(t, 7);
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
-            // the ring entry of this tile (row prefixes, carry, row-total accumulator, barriers) may be reused
-            mbar_arrive(smem_u32(&ctl->tot_empty[ts]));
+            // the carry ring entry of this tile (row prefixes, carry, barriers) may be reused
+            mbar_arrive(smem_u32(&ctl->ring_free[ts]));
         }
-        if (lane == 0) bulk_wait_all();
+        if (lane == 0 && wq == 0) PROF_FLUSH(32 + 8 * group, 6);
     }
 
     // ---- tear-down
