@@ -123,6 +123,13 @@ tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t 
  * `d_ws` since its last init gave up a bounded wait (its output is then not valid). */
 tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream);
 
+/* Self-test of the failure path (no counterpart in the paper): launches one warp that waits,
+ * for at most `limit_ms` milliseconds (1..1000), on a tile record that nothing publishes, and
+ * then records the time-out in the workspace header the way the scan kernels do.  After the
+ * stream has drained, tcu_scan_device_status(d_ws) returns TCU_ERR_TIMEOUT and the context is
+ * still usable; tcu_scan_workspace_init() clears the condition.  Nothing faults or hangs. */
+tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned limit_ms, cudaStream_t stream);
+
 /* Copies the bookkeeping of the most recent scan call made by this process. */
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out);
 

@@ -47,6 +47,8 @@ _lib.tcu_scan_host.argtypes = [_vp, _vp, _sz, _int, _int, _int, _vp, _vp, _vp, _
 _lib.tcu_scan_host.restype = _int
 _lib.tcu_scan_device_status.argtypes = [_vp, _vp]
 _lib.tcu_scan_device_status.restype = _int
+_lib.tcu_scan_selftest_timeout.argtypes = [_vp, _sz, ctypes.c_uint, _vp]
+_lib.tcu_scan_selftest_timeout.restype = _int
 _lib.tcu_scan_last_stats.argtypes = [ctypes.POINTER(TcuScanStats)]
 _lib.tcu_scan_last_stats.restype = _int
 _lib.tcu_status_string.argtypes = [_int]
@@ -99,6 +101,10 @@ def tcu_scan_host(h_in, h_out, n: int, dt: int, s: int, exclusive: int, d_in, d_
 
 def tcu_scan_device_status(d_ws, stream=0) -> int:
     return _lib.tcu_scan_device_status(_p(d_ws), stream)
+
+
+def tcu_scan_selftest_timeout(d_ws, ws_bytes: int, limit_ms: int, stream=0) -> int:
+    return _lib.tcu_scan_selftest_timeout(_p(d_ws), ws_bytes, int(limit_ms), stream)
 
 
 def tcu_scan_last_stats() -> dict:

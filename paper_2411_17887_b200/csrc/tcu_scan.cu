@@ -273,6 +273,14 @@ tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream) {
     return h.error == 0 ? TCU_OK : TCU_ERR_TIMEOUT;
 }
 
+tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned limit_ms, cudaStream_t stream) {
+    if (!d_ws || ws_bytes < size_t(kHeaderBytes) + 16) return TCU_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
+    if (limit_ms == 0 || limit_ms > 1000) return TCU_ERR_INVALID_ARG;
+    tcu_scan_timeout_selftest_kernel<<<1, 32, 0, stream>>>(d_ws, (long long)limit_ms * 2000000LL);
+    return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+}
+
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out) {
     if (!out) return TCU_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(g_stats_mutex);

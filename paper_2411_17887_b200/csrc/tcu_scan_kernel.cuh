@@ -1,21 +1,20 @@
 // Single-pass tensor-core-unit scan for sm_100a: device code.
 //
 // One persistent CTA per SM processes 128 x 128-element tiles.  Roles (warps):
-//   0      TMA producer: claims the next tile and loads it into a shared-memory ring
-//   1      MMA issuer, local scans: tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into one of
-//          three TMEM accumulators (Algorithm 1, up-sweep round t = 0: every length-s chunk becomes
-//          its own scan)
-//   2      MMA issuer, row totals: tcgen05.mma  R[128 x 16] = X[128 x 128] * ones  into a ring of
-//          eight small TMEM accumulators, issued as soon as the tile has landed - long before a
-//          full accumulator is free - so that the cross-tile carry scan starts early
-//   3      idle
-//   4-11   carry add and store (two groups of four warps taking alternate tiles): add chunk, row
-//          and tile carries to every element on the vector ALUs (down-sweep; the paper's
-//          discussion section recommends a vector unit for this add), stage the result in
-//          swizzled shared memory, write it with TMA stores
-//   12-15  totals: scan the 128 row totals (up-sweep rounds t >= 1), publish the tile total
-//   16-19  carry scan across tiles: decoupled look-back over per-tile records in global memory
-//          (Section 2.2 steps 2-3: totals of the segments, and their scan)
+//   0        TMA producer: claims the next tile and loads it into a shared-memory ring
+//   1        MMA issuer, local scans: tcgen05.mma  D[128 x 128] = X[128 x 128] * (I (x) U_s)  into one of
+//            three TMEM accumulators (Algorithm 1, up-sweep round t = 0: every length-s chunk
+//            becomes its own scan)
+//   2        MMA issuer, row totals: tcgen05.mma  R[128 x 16] = X[128 x 128] * ones  into a ring of
+//            eight small TMEM accumulators, issued as soon as the tile has landed - long before a
+//            full accumulator is free - so that the cross-tile carry scan starts early
+//   12-15    totals: scan the 128 row totals (up-sweep rounds t >= 1), publish the tile total
+//   3, 16-19 carry scan across tiles: decoupled look-back over per-tile records in global memory
+//            (Section 2.2 steps 2-3: totals of the segments, and their scan)
+//   4-11     carry add and store (two groups of four warps taking alternate tiles): add chunk, row
+//            and tile carries to every element on the vector ALUs (down-sweep; the paper's
+//            discussion section recommends a vector unit for this add), transpose through a
+//            swizzled shared-memory slab, write whole 128-byte lines with st.global.v4
 // Every wait is bounded; a wait that runs out records TCU_ERR_TIMEOUT in the workspace
 // header, and the CTA winds down (drains its copies, frees TMEM) instead of spinning.
 #pragma once
@@ -60,9 +59,7 @@ constexpr int kNumMarkers = kNumLookbackWarps;   // markers pushed: one per look
 #define TCU_PIPE_STORE 0
 #endif
 constexpr int kMaxInStages = 12;        // size of the barrier arrays
-constexpr int kUseInStages = TCU_MAX_STAGES;   // stages actually used: a tile is claimed when a stage frees, and claiming
-                                        // earlier than its row-total slot frees (kNumTot - kNumAcc tiles ahead) only
-                                        // makes later tiles of other CTAs wait for it
+constexpr int kUseInStages = TCU_MAX_STAGES;   // most stages the host will ask for
 constexpr int kLookBack = TCU_LOOKBACK; // records fetched per lane and round of the cross-tile look-back
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
@@ -882,6 +879,27 @@ __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start, ui
         if (IS_INT) reinterpret_cast<uint32_t *>(out)[start + tid] = uint32_t(y);
         else reinterpret_cast<float *>(out)[start + tid] = float(y);
     }
+}
+
+// Self-test of the bounded wait: one warp polls a tile record that nothing publishes, with a short
+// limit, records TCU_ERR_TIMEOUT in the workspace header exactly as the scan kernel does, and returns.
+__global__ void tcu_scan_timeout_selftest_kernel(void *ws, long long limit_cycles) {
+    WsHeader *hdr = reinterpret_cast<WsHeader *>(ws);
+    const uint8_t *rec = reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes;
+    const uint32_t epoch = ld_relaxed_u32(&hdr->epoch) + 1;     // a launch that never happens
+    uint64_t flag = 0, val = 0;
+    const long long c0 = clock64();
+    bool gave_up = false;
+    while (true) {
+        __nanosleep(100);
+        ld_record(rec, flag, val);
+        if (static_cast<uint32_t>(flag >> 2) == epoch) break;
+        if (clock64() - c0 > limit_cycles) {
+            gave_up = true;
+            break;
+        }
+    }
+    if (__any_sync(0xffffffffu, gave_up) && threadIdx.x == 0) atomicExch(&hdr->error, 5u);
 }
 
 }  // namespace tcu
