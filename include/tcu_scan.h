@@ -48,7 +48,8 @@ typedef enum {
     TCU_ERR_UNSUPPORTED = 2, /* valid request the library does not implement (see each call)      */
     TCU_ERR_WORKSPACE = 3,   /* workspace missing or smaller than tcu_scan_workspace_bytes()       */
     TCU_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (no device, launch failure...) */
-    TCU_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out; the output is not valid        */
+    TCU_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out; the output is not valid        */
+    TCU_ERR_TOO_LARGE = 6    /* tcu_scan_inclusive_noalloc: n exceeds TCU_SCAN_NOALLOC_MAX_ELEMENTS */
 } tcu_status_t;
 
 /* input element type -> output element type */
@@ -91,6 +92,31 @@ tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t s
  *   d_ws   device workspace of at least tcu_scan_workspace_bytes(1, n, dt, s) bytes */
 tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                 void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Inclusive scan for callers that cannot hand the library a workspace.  (The paper has no
+ * counterpart for this entry point; it exists for integration reasons only.)
+ *
+ * Some callers have no way to allocate device memory at the moment they need a scan: a plug-in
+ * that lives inside a host program which carved up the GPU's memory at start-up and forbids
+ * cudaMalloc afterwards (it would stall the device and may fail under a fixed budget), or a
+ * routine on a hot path that must not take the allocator's lock.  For them the tile records of
+ * the cross-tile carry scan live in a fixed array that is part of the library image itself.
+ * The caller still passes the input and the output; the call allocates and frees nothing.
+ *
+ *   n       at most TCU_SCAN_NOALLOC_MAX_ELEMENTS, else TCU_ERR_TOO_LARGE (nothing is launched)
+ *   others  as for tcu_scan_inclusive
+ *
+ * Cost: every GPU on which the library is loaded holds about 64 KiB for the array until the
+ * process ends, whether this entry point is used or not.
+ * First use: the first call on each device looks up the array's device address (that device
+ * must be current); make that first call before starting any stream capture.
+ * Sharing: there is one array per device and every call uses it, so two calls whose kernels
+ * could overlap on the GPU (different streams, no dependency between them) corrupt each
+ * other's carries; serialise them.  Each call clears the part of the array it needs, on
+ * `stream`, before its kernel runs. */
+#define TCU_SCAN_NOALLOC_MAX_ELEMENTS (1u << 26)
+tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
+                                        cudaStream_t stream);
 
 /* Exclusive scan, y[0] = 0, y[i] = x[0] + ... + x[i-1]  (the paper names the exclusive
  * form only in Table 1; this is the standard reading: shifted by one, identity 0 in front).

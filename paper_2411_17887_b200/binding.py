@@ -11,7 +11,8 @@ import os
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libtcu_scan.so")
 
-TCU_OK, TCU_ERR_INVALID_ARG, TCU_ERR_UNSUPPORTED, TCU_ERR_WORKSPACE, TCU_ERR_CUDA, TCU_ERR_TIMEOUT = range(6)
+TCU_OK, TCU_ERR_INVALID_ARG, TCU_ERR_UNSUPPORTED, TCU_ERR_WORKSPACE, TCU_ERR_CUDA, TCU_ERR_TIMEOUT, TCU_ERR_TOO_LARGE = range(7)
+TCU_SCAN_NOALLOC_MAX_ELEMENTS = 1 << 26
 TCU_I8_I32, TCU_F16_F32, TCU_BF16_F32 = range(3)
 DTYPES = {"i8": TCU_I8_I32, "f16": TCU_F16_F32, "bf16": TCU_BF16_F32}
 
@@ -41,6 +42,8 @@ _lib.tcu_scan_workspace_init.restype = _int
 for _name in ("tcu_scan_inclusive", "tcu_scan_exclusive", "tcu_scan_level0_debug"):
     getattr(_lib, _name).argtypes = [_vp, _vp, _sz, _int, _int, _vp, _sz, _vp]
     getattr(_lib, _name).restype = _int
+_lib.tcu_scan_inclusive_noalloc.argtypes = [_vp, _vp, _sz, _int, _int, _vp]
+_lib.tcu_scan_inclusive_noalloc.restype = _int
 _lib.tcu_scan_batched.argtypes = [_vp, _vp, _sz, _sz, _int, _int, _int, _vp, _sz, _vp]
 _lib.tcu_scan_batched.restype = _int
 _lib.tcu_scan_host.argtypes = [_vp, _vp, _sz, _int, _int, _int, _vp, _vp, _vp, _sz, _vp]
@@ -78,6 +81,12 @@ def tcu_scan_workspace_init(d_ws, ws_bytes: int, stream=0) -> int:
 
 def tcu_scan_inclusive(d_in, d_out, n: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0) -> int:
     return _lib.tcu_scan_inclusive(_p(d_in), _p(d_out), n, dt, s, _p(d_ws), ws_bytes, stream)
+
+
+def tcu_scan_inclusive_noalloc(d_in, d_out, n: int, dt: int, s: int, stream=0) -> int:
+    """Inclusive scan that takes no workspace: the carry records live in an array built into the
+    library (at most TCU_SCAN_NOALLOC_MAX_ELEMENTS elements; calls must not overlap on the GPU)."""
+    return _lib.tcu_scan_inclusive_noalloc(_p(d_in), _p(d_out), n, dt, s, stream)
 
 
 def tcu_scan_exclusive(d_in, d_out, n: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0) -> int:

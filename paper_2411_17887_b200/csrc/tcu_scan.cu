@@ -217,6 +217,31 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     return TCU_OK;
 }
 
+// Built-in scratch of tcu_scan_inclusive_noalloc: the tile records of the cross-tile carry scan for
+// at most TCU_SCAN_NOALLOC_MAX_ELEMENTS elements.  One copy per GPU that loads this library, held
+// until the process exits.  In host code this name is only a handle for the runtime: the address the
+// kernels need comes from cudaGetSymbolAddress (see noalloc_scratch below).
+constexpr size_t kNoAllocScratchBytes =
+    size_t(kHeaderBytes) + 16 * (size_t(TCU_SCAN_NOALLOC_MAX_ELEMENTS) / kTileElems) + 16;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+// Device address of the built-in scratch on the current device, looked up once per device.
+tcu_status_t noalloc_scratch(void **out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void *addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TCU_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return TCU_ERR_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return TCU_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -236,6 +261,20 @@ tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t s
 tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
                                 size_t ws_bytes, cudaStream_t stream) {
     return scan_impl(d_in, d_out, 1, n, dt, s, false, false, d_ws, ws_bytes, stream);
+}
+
+tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
+                                        cudaStream_t stream) {
+    if (n > size_t(TCU_SCAN_NOALLOC_MAX_ELEMENTS)) return TCU_ERR_TOO_LARGE;
+    if (n == 0) return TCU_OK;
+    void *scratch = nullptr;
+    tcu_status_t st = noalloc_scratch(&scratch);
+    if (st != TCU_OK) return st;
+    // The scratch still holds the records of whatever call used it last.  Everything the kernels
+    // expect to find at zero (header counters, the records of this call's tiles) is cleared here.
+    const size_t used = tcu_scan_workspace_bytes(1, n, dt, s);
+    if (cudaMemsetAsync(scratch, 0, used, stream) != cudaSuccess) return TCU_ERR_CUDA;
+    return scan_impl(d_in, d_out, 1, n, dt, s, false, false, scratch, kNoAllocScratchBytes, stream);
 }
 
 tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
@@ -309,6 +348,7 @@ const char *tcu_status_string(tcu_status_t st) {
         case TCU_ERR_WORKSPACE: return "workspace missing or too small";
         case TCU_ERR_CUDA: return "CUDA call failed";
         case TCU_ERR_TIMEOUT: return "device-side wait timed out";
+        case TCU_ERR_TOO_LARGE: return "problem larger than the built-in scratch allows";
         default: return "unknown status";
     }
 }
