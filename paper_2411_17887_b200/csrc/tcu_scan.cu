@@ -177,6 +177,15 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
         }
+        {
+            const cuuint64_t strides[2] = {cuuint64_t(kTileCols) * 4, pitch_elems * 4};
+            const cuuint32_t box[3] = {32, 32, 1};   // one slab: 32 columns x 32 rows, stored by one warp
+            CUtensorMapDataType ty = dt == TCU_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+            CUresult r = encode(&prm.tmap_out, ty, 3, d_out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
+        }
         prm.ws = d_ws;
         prm.out = d_out;
         prm.scan_pitch = cols;

@@ -29,6 +29,15 @@ namespace tcu {
 #ifndef TCU_STORE_GROUPS
 #define TCU_STORE_GROUPS 2
 #endif
+#ifndef TCU_PREFETCH_DIST
+#define TCU_PREFETCH_DIST 256
+#endif
+#ifndef TCU_TMA_STORE
+#define TCU_TMA_STORE 0
+#endif
+#ifndef TCU_SETMAXNREG
+#define TCU_SETMAXNREG 1
+#endif
 #ifndef TCU_LOOKBACK
 #define TCU_LOOKBACK 2
 #endif
@@ -46,7 +55,11 @@ constexpr int kTotBase = kNumAcc * kTileCols;            // first TMEM column of
 static_assert(kTotBase + kNumTot * kTotCols <= 512, "TMEM has 512 columns");
 constexpr int kStoreGroups = TCU_STORE_GROUPS;           // groups of 4 store warps; group g takes the tiles with j % kStoreGroups == g
 constexpr int kSlabBytes = 32 * 4 * 32;                  // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
-constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabBytes;   // one transposition slab per store warp
+#ifndef TCU_SLABS
+#define TCU_SLABS 2
+#endif
+constexpr int kSlabsPerWarp = TCU_TMA_STORE ? TCU_SLABS : 1;   // TMA stores read the slab asynchronously: ring of slabs
+constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabsPerWarp * kSlabBytes;   // staging slabs of the store warps
 constexpr int kNumCarry = 16;           // tiles a CTA may have between "row totals known" and "stored": ring of carry entries
 constexpr int kTileRing = 32;           // ring of claimed tile numbers (must exceed the tiles a CTA has in flight)
 constexpr uint32_t kNoTile = 0xFFFFFFFFu;   // "no more tiles" marker pushed through the pipeline
@@ -60,10 +73,16 @@ constexpr int kNumMarkers = kNumLookbackWarps;   // markers pushed: one per look
 #endif
 constexpr int kMaxInStages = 12;        // size of the barrier arrays
 constexpr int kUseInStages = TCU_MAX_STAGES;   // most stages the host will ask for
+constexpr uint32_t kPrefetchDist = TCU_PREFETCH_DIST;   // tiles ahead of the claimed one that are prefetched into L2
 constexpr int kLookBack = TCU_LOOKBACK; // records fetched per lane and round of the cross-tile look-back
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
 constexpr int kEpilogueThreads = 128;
+// Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
+// 96 x 640 = 61440 registers), so 128 x (64 + 64 + 40 + kStoreGroups x kStoreRegs) must not exceed it:
+// an increase that cannot be granted would block.
+constexpr int kStoreRegs = (kStoreGroups == 3) ? 104 : 128;
+static_assert(128 * (64 + 64 + 40 + kStoreGroups * kStoreRegs) <= 61440, "register pool");
 constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back
@@ -112,6 +131,7 @@ constexpr long long kSpinLimitCycles = 2000000000LL;   // about one second at B2
 
 struct alignas(64) ScanParams {
     CUtensorMap tmap_in;      // (128, rows128, batch) view of the input, box 128 B x 128 rows
+    CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 32 (used by the TMA-store variant)
     void *ws;
     void *out;                // output array (4-byte elements)
     uint64_t scan_pitch;      // elements between consecutive scans (batched), unused for a single array
@@ -185,6 +205,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
+// Ask the TMA unit to bring a box into L2 only (no shared-memory destination, no completion signal).
+__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int x, int y, int z) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int x, int y, int z) {
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                  ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z)
@@ -209,6 +235,20 @@ __device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred)
         : "r"(uint32_t(pred)), "r"(id), "r"(threads)
         : "memory");
     return res != 0;
+}
+// Register re-allocation between warpgroups (4 consecutive warps): the store warps need many
+// registers, every other role few.  All four warps of a group must execute the same instruction.
+template <int N>
+__device__ __forceinline__ void reg_dec() {
+#if TCU_SETMAXNREG
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+#endif
+}
+template <int N>
+__device__ __forceinline__ void reg_inc() {
+#if TCU_SETMAXNREG
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+#endif
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -444,132 +484,12 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     // whoever holds tile t knows that every tile before t is held by a CTA that is already running).  When
     // the tiles run out the producer pushes kNumMarkers "no more tiles" markers through the pipeline, so
     // that every role - and each of the look-back warps - sees one and stops.
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t issued = 0, markers = 0;
-            PROF_DECL
-            PROF_T0();
-            for (uint32_t j = 0;; ++j) {
-                uint32_t stage = j % num_in, u = j / num_in;
-                if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
-                PROF_ADD(0);
-                uint32_t t = kNoTile;
-                if (markers == 0) t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
-                if (t >= p.tiles_total) t = kNoTile;
-                PROF_ADD(1);
-                PROF_INC(3, 1);
-                ctl->tile_of[j % kTileRing] = t;
-                uint32_t bar = smem_u32(&ctl->full[stage]);
-                if (t == kNoTile) {
-                    mbar_arrive(bar);
-                    if (++markers == kNumMarkers) break;
-                    continue;
-                }
-                TRACE(t, 0);
-                mbar_expect_tx(bar, kStageBytes);
-                int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
-#pragma unroll
-                for (int a = 0; a < kInAtoms; ++a)
-                    tma_load_3d(smem_u32(in_ring + stage * kStageBytes + a * kAtomBytes), &p.tmap_in,
-                                a * (128 / kElemBytes), lt * kTileRows, scan_row, bar);
-                issued = j + 1;
-                PROF_ADD(2);
-            }
-            PROF_FLUSH(0, 4);
-            if (ctl->abort_flag) {
-                // drain: loads already issued must land before the CTA may exit
-                uint32_t lo = issued > num_in ? issued - num_in : 0;
-                for (uint32_t j = lo; j < issued; ++j) {
-                    uint32_t bar = smem_u32(&ctl->full[j % num_in]);
-                    uint32_t par = (j / num_in) & 1;
-                    long long t0 = clock64();
-                    while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinLimitCycles) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer: local scans
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(p.dtype, kSeff);
-            const uint32_t b_base = smem_u32(const_region);
-            uint32_t markers = 0;
-            PROF_DECL
-            PROF_T0();
-            for (uint32_t j = 0;; ++j) {
-                uint32_t stage = j % num_in, u = j / num_in;
-                uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
-                if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
-                PROF_ADD(0);
-                if (ctl->tile_of[j % kTileRing] == kNoTile) {
-                    mbar_arrive(smem_u32(&ctl->empty[stage]));
-                    if (++markers == kNumMarkers) break;
-                    continue;
-                }
-                if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
-                PROF_ADD(1);
-                tc_fence_after();
-                const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
-#pragma unroll
-                for (int g = 0; g < kSegs; ++g) {
-#pragma unroll
-                    for (int kk = 0; kk < kKSteps; ++kk) {
-                        int a_off = (g * kKSteps + kk) * 32;
-                        int b_off = kk * 32;
-                        uint64_t adesc = make_smem_desc(a_base + (a_off >> 7) * kAtomBytes + (a_off & 127));
-                        uint64_t bdesc = make_smem_desc(b_base + (b_off >> 7) * kAtomBytes + (b_off & 127));
-                        mma_issue<IS_INT>(tmem_base + slot * kTileCols + g * kSeff, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
-                    }
-                }
-                mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once both issuers' MMAs have read it
-                mma_commit(smem_u32(&ctl->acc_full[slot]));
-                PROF_ADD(2);
-            }
-            PROF_FLUSH(4, 3);
-        }
-    } else if (warp == 2) {
-        // ------------------------------------------------------------------ MMA issuer: row totals
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(p.dtype, kTotCols);
-            const uint64_t bdesc = make_smem_desc(smem_u32(ones_region));
-            uint32_t markers = 0;
-            PROF_DECL
-            PROF_T0();
-            for (uint32_t j = 0;; ++j) {
-                uint32_t stage = j % num_in, u = j / num_in;
-                uint32_t ts = j % kNumTot, ut = j / kNumTot;
-                if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
-                PROF_ADD(0);
-                if (!w.wait(smem_u32(&ctl->tot_empty[ts]), (ut & 1) ^ 1)) break;
-                PROF_ADD(1);
-                if (ctl->tile_of[j % kTileRing] == kNoTile) {
-                    mbar_arrive(smem_u32(&ctl->empty[stage]));
-                    mbar_arrive(smem_u32(&ctl->tot_full[ts]));
-                    if (++markers == kNumMarkers) break;
-                    continue;
-                }
-                TRACE(ctl->tile_of[j % kTileRing], 1);
-                TRACE_V(ctl->tile_of[j % kTileRing], 2, blockIdx.x);
-                tc_fence_after();
-                const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
-#pragma unroll
-                for (int kk = 0; kk < kRowKSteps; ++kk) {
-                    int a_off = kk * 32;
-                    uint64_t adesc = make_smem_desc(a_base + (a_off >> 7) * kAtomBytes + (a_off & 127));
-                    mma_issue<IS_INT>(tmem_base + kTotBase + ts * kTotCols, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
-                }
-                mma_commit(smem_u32(&ctl->empty[stage]));
-                mma_commit(smem_u32(&ctl->tot_full[ts]));
-                PROF_ADD(2);
-            }
-            PROF_FLUSH(8, 3);
-        }
-    } else if (warp == 3 || warp >= kFirstLookbackWarp) {
+    // ------------------------------------------------------------------ cross-tile carry scan (role of warp 3 and warps 20-23)
+    auto lookback_role = [&](const uint32_t lbw) {
         // ------------------------------------------------------------------ cross-tile carry scan
         // kNumLookbackWarps warps take the tiles in turn, so that the look-backs of the tiles in flight overlap.
         PROF_DECL
         PROF_T0();
-        const uint32_t lbw = (warp == 3) ? 0u : uint32_t(warp - kFirstLookbackWarp + 1);
         for (uint32_t j = lbw;; j += kNumLookbackWarps) {
             const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;
             if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[ts]), ut & 1))) break;
@@ -659,7 +579,147 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             PROF_INC(3, 1);
         }
         if (lane == 0) PROF_FLUSH(12 + 4 * (lbw % 4), 4);
+    };
+
+    if (warp < 4) {
+    reg_dec<64>();                                     // producer, MMA issuers, one look-back warp
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t issued = 0, markers = 0;
+            PROF_DECL
+            PROF_T0();
+            for (uint32_t j = 0;; ++j) {
+                uint32_t stage = j % num_in, u = j / num_in;
+                if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
+                PROF_ADD(0);
+                uint32_t t = kNoTile;
+                if (markers == 0) t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
+                if (t >= p.tiles_total) t = kNoTile;
+                PROF_ADD(1);
+                PROF_INC(3, 1);
+                ctl->tile_of[j % kTileRing] = t;
+                uint32_t bar = smem_u32(&ctl->full[stage]);
+                if (t == kNoTile) {
+                    mbar_arrive(bar);
+                    if (++markers == kNumMarkers) break;
+                    continue;
+                }
+                TRACE(t, 0);
+                mbar_expect_tx(bar, kStageBytes);
+                int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
+#pragma unroll
+                for (int a = 0; a < kInAtoms; ++a)
+                    tma_load_3d(smem_u32(in_ring + stage * kStageBytes + a * kAtomBytes), &p.tmap_in,
+                                a * (128 / kElemBytes), lt * kTileRows, scan_row, bar);
+                issued = j + 1;
+                // Tiles are claimed in increasing order by all CTAs, so tile t + kPrefetchDist will be claimed by
+                // somebody a few microseconds from now: start its trip from DRAM to L2 now.  Its later load then
+                // costs an L2 hit, which takes the DRAM latency - and its spread - out of the carry chain.
+                if (kPrefetchDist > 0 && t + kPrefetchDist < p.tiles_total) {
+                    const uint32_t tp = t + kPrefetchDist;
+                    const int prow = tp / p.tiles_per_row, plt = tp % p.tiles_per_row;
+#pragma unroll
+                    for (int a = 0; a < kInAtoms; ++a)
+                        tma_prefetch_l2_3d(&p.tmap_in, a * (128 / kElemBytes), plt * kTileRows, prow);
+                }
+                PROF_ADD(2);
+            }
+            PROF_FLUSH(0, 4);
+            if (ctl->abort_flag) {
+                // drain: loads already issued must land before the CTA may exit
+                uint32_t lo = issued > num_in ? issued - num_in : 0;
+                for (uint32_t j = lo; j < issued; ++j) {
+                    uint32_t bar = smem_u32(&ctl->full[j % num_in]);
+                    uint32_t par = (j / num_in) & 1;
+                    long long t0 = clock64();
+                    while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinLimitCycles) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer: local scans
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(p.dtype, kSeff);
+            const uint32_t b_base = smem_u32(const_region);
+            uint32_t markers = 0;
+            PROF_DECL
+            PROF_T0();
+            for (uint32_t j = 0;; ++j) {
+                uint32_t stage = j % num_in, u = j / num_in;
+                uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
+                if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                PROF_ADD(0);
+                if (ctl->tile_of[j % kTileRing] == kNoTile) {
+                    mbar_arrive(smem_u32(&ctl->empty[stage]));
+                    if (++markers == kNumMarkers) break;
+                    continue;
+                }
+                if (!w.wait(smem_u32(&ctl->acc_empty[slot]), (ua & 1) ^ 1)) break;
+                PROF_ADD(1);
+                tc_fence_after();
+                const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
+#pragma unroll
+                for (int g = 0; g < kSegs; ++g) {
+#pragma unroll
+                    for (int kk = 0; kk < kKSteps; ++kk) {
+                        int a_off = (g * kKSteps + kk) * 32;
+                        int b_off = kk * 32;
+                        uint64_t adesc = make_smem_desc(a_base + (a_off >> 7) * kAtomBytes + (a_off & 127));
+                        uint64_t bdesc = make_smem_desc(b_base + (b_off >> 7) * kAtomBytes + (b_off & 127));
+                        mma_issue<IS_INT>(tmem_base + slot * kTileCols + g * kSeff, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                    }
+                }
+                mma_commit(smem_u32(&ctl->empty[stage]));      // the stage may be refilled once both issuers' MMAs have read it
+                mma_commit(smem_u32(&ctl->acc_full[slot]));
+                PROF_ADD(2);
+            }
+            PROF_FLUSH(4, 3);
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ MMA issuer: row totals
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(p.dtype, kTotCols);
+            const uint64_t bdesc = make_smem_desc(smem_u32(ones_region));
+            uint32_t markers = 0;
+            PROF_DECL
+            PROF_T0();
+            for (uint32_t j = 0;; ++j) {
+                uint32_t stage = j % num_in, u = j / num_in;
+                uint32_t ts = j % kNumTot, ut = j / kNumTot;
+                if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
+                PROF_ADD(0);
+                if (!w.wait(smem_u32(&ctl->tot_empty[ts]), (ut & 1) ^ 1)) break;
+                PROF_ADD(1);
+                if (ctl->tile_of[j % kTileRing] == kNoTile) {
+                    mbar_arrive(smem_u32(&ctl->empty[stage]));
+                    mbar_arrive(smem_u32(&ctl->tot_full[ts]));
+                    if (++markers == kNumMarkers) break;
+                    continue;
+                }
+                TRACE(ctl->tile_of[j % kTileRing], 1);
+                tc_fence_after();
+                const uint32_t a_base = smem_u32(in_ring + stage * kStageBytes);
+#pragma unroll
+                for (int kk = 0; kk < kRowKSteps; ++kk) {
+                    int a_off = kk * 32;
+                    uint64_t adesc = make_smem_desc(a_base + (a_off >> 7) * kAtomBytes + (a_off & 127));
+                    mma_issue<IS_INT>(tmem_base + kTotBase + ts * kTotCols, adesc, bdesc, idesc, kk > 0 ? 1u : 0u);
+                }
+                mma_commit(smem_u32(&ctl->empty[stage]));
+                mma_commit(smem_u32(&ctl->tot_full[ts]));
+                PROF_ADD(2);
+            }
+            PROF_FLUSH(8, 3);
+        }
+    } else {
+        lookback_role(0);
+    }
+    } else if (warp >= kFirstLookbackWarp) {
+        reg_dec<64>();
+        lookback_role(uint32_t(warp - kFirstLookbackWarp + 1));
     } else if (warp >= kFirstTotalsWarp) {
+        reg_dec<40>();
         // ------------------------------------------------------------------ totals (up-sweep above the product)
         // Takes the 128 row totals from the small accumulator, scans them across the rows, and
         // publishes the tile total - as soon as the tile has landed, so that the cross-tile look-back
@@ -685,6 +745,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (++markers == kNumMarkers) break;
                 continue;
             }
+            if (r == 0) TRACE(t, 2);
             tc_fence_after();
             const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
             tmem_ld_wait();
@@ -722,7 +783,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             PROF_ADD(1);
         }
         if (r == 0) PROF_FLUSH(28, 2);
-    } else if (warp >= kFirstStoreWarp) {
+    } else {
+        reg_inc<kStoreRegs>();
         // ------------------------------------------------------------------ carry add and store (down-sweep)
         // Every warp works alone on its 32 rows: TMEM -> registers (one row per lane) -> add carries ->
         // swizzled 4 KB slab in shared memory -> read back with eight lanes per row -> st.global.v4,
@@ -731,7 +793,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const int wq = warp & 3;                                    // TMEM lane quarter this warp may read
         const int r = wq * 32 + lane;                               // tile row owned by this thread
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
-        const uint32_t slab = smem_u32(out_ring) + (warp - kFirstStoreWarp) * kSlabBytes;
+        const uint32_t slab0 = smem_u32(out_ring) + (warp - kFirstStoreWarp) * kSlabsPerWarp * kSlabBytes;
+        uint32_t slab_counter = 0;
+        (void)slab_counter;
         const int sub = lane >> 3, piece = lane & 7;                // read-back role: row sub (+4i) of the slab, 16-byte piece
         uint32_t *const out32 = reinterpret_cast<uint32_t *>(p.out);
         PROF_DECL
@@ -786,6 +850,24 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 }
                 // fetch the next 32 columns while this chunk is transposed and stored
                 if (TCU_PIPE_STORE && q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
+#if TCU_TMA_STORE
+                if (lane == 0) bulk_wait_read<kSlabsPerWarp - 1>();    // the slab about to be written has been drained
+                __syncwarp();
+                const uint32_t slab = slab0 + (slab_counter % kSlabsPerWarp) * kSlabBytes;
+                const uint32_t buf = slab + lane * 128;
+#pragma unroll
+                for (int c4 = 0; c4 < 8; ++c4)
+                    st_shared_v4(buf + ((c4 ^ (lane & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                PROF_ADD(3);
+                if (lane == 0) {
+                    tma_store_3d(&p.tmap_out, slab, q * 32, row0, scan_row);
+                    bulk_commit();
+                }
+                ++slab_counter;
+#else
+                const uint32_t slab = slab0;
                 __syncwarp();                                         // the slab has been read back by every lane
                 const uint32_t buf = slab + lane * 128;
 #pragma unroll
@@ -805,6 +887,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     if (rr < rows_here)
                         st_global_v4(gbase + size_t(rr) * kTileCols + q * 32, a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
                 }
+#endif
                 PROF_ADD(4);
                 if (!TCU_PIPE_STORE && q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
             }
@@ -814,6 +897,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             // the carry ring entry of this tile (row prefixes, carry, barriers) may be reused
             mbar_arrive(smem_u32(&ctl->ring_free[ts]));
         }
+        if (TCU_TMA_STORE && lane == 0) bulk_wait_all();
         if (lane == 0 && wq == 0) PROF_FLUSH(32 + 8 * group, 6);
     }
 
