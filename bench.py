@@ -32,7 +32,7 @@ BYTES_PER_ELEM = 5          # int8 read + int32 written
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel, from the ncu
 # capture summarised in profiles/ (scaled to a full launch as described there); None until captured
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 277.15e6   # profiles/tcu_scan_kernel_int8_s16_n2p26_ncu_full.md, scaled x4 to n = 2^28
 
 
 def measured_peak():
