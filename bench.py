@@ -131,12 +131,14 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def time_extra(B, torch, name, x, rows, cols, dt, s, exclusive, ws_ptr, ws_bytes, reps=10):
+def time_extra(B, torch, name, x, rows, cols, dt, s, exclusive, ws_ptr, ws_bytes, reps=10, two_sweep=False):
     out = torch.empty(rows * cols, dtype=torch.int32 if dt == 0 else torch.float32, device="cuda")
     stream = torch.cuda.current_stream().cuda_stream
 
     def call():
-        if rows == 1:
+        if two_sweep:
+            B.check(B.tcu_scan_inclusive_twosweep(x, out, cols, dt, s, ws_ptr, ws_bytes, stream))
+        elif rows == 1:
             fn = B.tcu_scan_exclusive if exclusive else B.tcu_scan_inclusive
             B.check(fn(x, out, cols, dt, s, ws_ptr, ws_bytes, stream))
         else:
@@ -284,6 +286,10 @@ def run_ours(args):
                 xb = torch.randn(1 << 28, device="cuda", generator=g).bfloat16()
                 extras.append(time_extra(B, torch, "C4: 4096 x 65536 bf16 normal -> fp32, s=16, row-wise", xb, 4096, 65536, 2, 16, False, ws_ptr, ws_bytes))
                 extras.append(time_extra(B, torch, "C1: n=2^16 int8, s=16", d_in, 1, 1 << 16, 0, 16, False, ws_ptr, ws_bytes))
+                extras.append(time_extra(B, torch, "C3 in the two-sweep structure (reduce, scan totals, scan): n=2^28 int8, s=16",
+                                         d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes, two_sweep=True))
+                extras.append(time_extra(B, torch, "fp16 n=2^28 in the two-sweep structure, s=16",
+                                         xf, 1, 1 << 28, 1, 16, False, ws_ptr, ws_bytes, two_sweep=True))
                 line["extra"] = extras
         print(json.dumps(line))
     if world > 1:

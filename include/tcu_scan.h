@@ -63,7 +63,7 @@ typedef enum {
 typedef struct {
     uint64_t rows, cols;        /* problem shape (rows = 1 for the single-array calls)               */
     uint32_t s, dtype, exclusive;
-    uint32_t variant;           /* 0 = single pass, decoupled look-back                              */
+    uint32_t variant;           /* 0 = single pass, decoupled look-back; 1 = two sweeps                 */
     uint32_t upper_level_path;  /* 0 = levels above the U_s product run on CUDA cores (warp shuffles)  */
     uint64_t tiles;             /* 128 x 128-element tiles processed                                  */
     uint64_t mma_instructions;  /* tcgen05.mma instructions issued                                    */
@@ -123,6 +123,15 @@ tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n,
  * Arguments as for tcu_scan_inclusive. */
 tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                 void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* The same inclusive scan in the two-sweep structure of classical work-efficient scans (the
+ * paper's up-sweep / down-sweep split across kernels): sweep 1 reads the input and reduces every
+ * tile to its total, a one-block kernel scans the totals, sweep 2 is the single-pass kernel with
+ * every carry already known.  It reads the input twice and exists so that the choice between
+ * the two structures can be measured; results satisfy the same parity bars.  Arguments as for
+ * tcu_scan_inclusive. */
+tcu_status_t tcu_scan_inclusive_twosweep(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
+                                         void *d_ws, size_t ws_bytes, cudaStream_t stream);
 
 /* `rows` independent scans of `cols` elements each, dense row-major (row stride = cols)
  * (Section 2.2 step 1: the algorithm run on each contiguous segment, no stitching).

@@ -39,7 +39,7 @@ _lib.tcu_scan_workspace_bytes.argtypes = [_sz, _sz, _int, _int]
 _lib.tcu_scan_workspace_bytes.restype = _sz
 _lib.tcu_scan_workspace_init.argtypes = [_vp, _sz, _vp]
 _lib.tcu_scan_workspace_init.restype = _int
-for _name in ("tcu_scan_inclusive", "tcu_scan_exclusive", "tcu_scan_level0_debug"):
+for _name in ("tcu_scan_inclusive", "tcu_scan_exclusive", "tcu_scan_level0_debug", "tcu_scan_inclusive_twosweep"):
     getattr(_lib, _name).argtypes = [_vp, _vp, _sz, _int, _int, _vp, _sz, _vp]
     getattr(_lib, _name).restype = _int
 _lib.tcu_scan_inclusive_noalloc.argtypes = [_vp, _vp, _sz, _int, _int, _vp]
@@ -87,6 +87,10 @@ def tcu_scan_inclusive_noalloc(d_in, d_out, n: int, dt: int, s: int, stream=0) -
     """Inclusive scan that takes no workspace: the carry records live in an array built into the
     library (at most TCU_SCAN_NOALLOC_MAX_ELEMENTS elements; calls must not overlap on the GPU)."""
     return _lib.tcu_scan_inclusive_noalloc(_p(d_in), _p(d_out), n, dt, s, stream)
+
+
+def tcu_scan_inclusive_twosweep(d_in, d_out, n: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0) -> int:
+    return _lib.tcu_scan_inclusive_twosweep(_p(d_in), _p(d_out), n, dt, s, _p(d_ws), ws_bytes, stream)
 
 
 def tcu_scan_exclusive(d_in, d_out, n: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0) -> int:

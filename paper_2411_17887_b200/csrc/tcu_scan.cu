@@ -102,7 +102,8 @@ bool overlaps(const void *a, size_t an, const void *b, size_t bn) {
 }
 
 tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
-                       bool exclusive, bool level0, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+                       bool exclusive, bool level0, void *d_ws, size_t ws_bytes, cudaStream_t stream,
+                       bool two_sweep = false) {
     if (!valid_dtype(dt) || !valid_s(s)) return (s > 0 && valid_dtype(dt)) ? TCU_ERR_UNSUPPORTED : TCU_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return TCU_OK;
     if (!d_in || !d_out) return TCU_ERR_INVALID_ARG;
@@ -141,7 +142,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     st.s = s;
     st.dtype = dt;
     st.exclusive = exclusive;
-    st.variant = 0;
+    st.variant = two_sweep ? 1 : 0;
     st.upper_level_path = 0;
     st.tiles = tiles;
     st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32);  // U_s products + row-total products
@@ -196,6 +197,19 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         prm.b_bytes = b_bytes;
         prm.dtype = uint32_t(dt);
         prm.level0_only = level0 ? 1u : 0u;
+        prm.prefilled = two_sweep ? 1u : 0u;
+        if (two_sweep) {
+            // sweep 1: one total per tile; then their scan, written as the records sweep 2 looks back over
+            const uint64_t valid = uint64_t(rows128) * kTileCols;
+            if (dt == TCU_I8_I32) {
+                tcu_tile_totals_kernel<true><<<unsigned(tiles), 256, 0, stream>>>(d_in, d_ws, valid, dt);
+                tcu_totals_scan_kernel<true><<<1, 1024, 0, stream>>>(d_ws, uint32_t(tiles));
+            } else {
+                tcu_tile_totals_kernel<false><<<unsigned(tiles), 256, 0, stream>>>(d_in, d_ws, valid, dt);
+                tcu_totals_scan_kernel<false><<<1, 1024, 0, stream>>>(d_ws, uint32_t(tiles));
+            }
+            if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+        }
         // persistent grid: every CTA must be resident at once (the carry chain waits on
         // lower-numbered tiles), so never more CTAs than SMs; one CTA fills an SM's shared memory
         dim3 grid(unsigned(tiles < uint64_t(sms) ? tiles : uint64_t(sms)));
@@ -284,6 +298,11 @@ tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n,
     const size_t used = tcu_scan_workspace_bytes(1, n, dt, s);
     if (cudaMemsetAsync(scratch, 0, used, stream) != cudaSuccess) return TCU_ERR_CUDA;
     return scan_impl(d_in, d_out, 1, n, dt, s, false, false, scratch, kNoAllocScratchBytes, stream);
+}
+
+tcu_status_t tcu_scan_inclusive_twosweep(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
+                                         size_t ws_bytes, cudaStream_t stream) {
+    return scan_impl(d_in, d_out, 1, n, dt, s, false, false, d_ws, ws_bytes, stream, true);
 }
 
 tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,

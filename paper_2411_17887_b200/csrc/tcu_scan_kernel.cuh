@@ -142,6 +142,7 @@ struct alignas(64) ScanParams {
     uint32_t b_bytes;         // shared memory reserved for the constant operand I (x) U_s
     uint32_t dtype;           // tcu_dtype_t
     uint32_t level0_only;     // debug: stop after the U_s product (no carries)
+    uint32_t prefilled;       // two-sweep variant: the records already hold every tile's inclusive sum
 };
 
 // shared-memory bookkeeping (lives at the 1024-aligned base of dynamic shared memory)
@@ -567,7 +568,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     }
                 }
                 // publish even after a give-up so that successors do not wait for this tile
-                if (lane == 0) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
+                if (lane == 0 && !p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
             }
             if (lane == 0) {
                 TRACE(t, 5);
@@ -773,7 +774,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
                 // the first tile of a scan has nothing before it: its total is already inclusive
                 const uint32_t status = (t % p.tiles_per_row == 0) ? kStatusInclusive : kStatusPartial;
-                st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(a));
+                if (!p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(a));
                 TRACE(t, 3);
                 ctl->agg_slot[ts] = CO::enc(a);
             }
@@ -962,6 +963,107 @@ __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start, ui
     if (tid < int(count)) {
         if (IS_INT) reinterpret_cast<uint32_t *>(out)[start + tid] = uint32_t(y);
         else reinterpret_cast<float *>(out)[start + tid] = float(y);
+    }
+}
+
+// ---- two-sweep variant (for comparison with the single pass): sweep 1 reduces every tile to its
+// total, a one-block scan turns the totals into inclusive sums and writes them as the records the main
+// kernel's look-back expects, sweep 2 is the main kernel, whose look-back then succeeds at once.
+template <bool IS_INT>
+__global__ void __launch_bounds__(256) tcu_tile_totals_kernel(const void *in, void *ws, uint64_t valid_elems, uint32_t dtype) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    __shared__ CarryT part[8];
+    const uint32_t t = blockIdx.x;
+    const uint64_t base = uint64_t(t) * kTileElems;
+    CarryT acc = CarryT(0);
+    if (IS_INT) {
+        const int4 *src = reinterpret_cast<const int4 *>(reinterpret_cast<const int8_t *>(in) + base);
+        int sum = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t idx = i * 256 + threadIdx.x;                   // 16-byte piece of the tile
+            if (base + uint64_t(idx) * 16 < valid_elems) {
+                int4 v = src[idx];
+                sum = __dp4a(v.x, 0x01010101, sum);
+                sum = __dp4a(v.y, 0x01010101, sum);
+                sum = __dp4a(v.z, 0x01010101, sum);
+                sum = __dp4a(v.w, 0x01010101, sum);
+            }
+        }
+        acc = CarryT(uint32_t(sum));
+    } else {
+        const int4 *src = reinterpret_cast<const int4 *>(reinterpret_cast<const uint16_t *>(in) + base);
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t idx = i * 256 + threadIdx.x;                   // 16-byte piece = 8 elements
+            if (base + uint64_t(idx) * 8 < valid_elems) {
+                int4 v = src[idx];
+                const uint32_t w[4] = {uint32_t(v.x), uint32_t(v.y), uint32_t(v.z), uint32_t(v.w)};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float lo, hi;
+                    if (dtype == 2) {
+                        lo = __uint_as_float(w[k] << 16);
+                        hi = __uint_as_float(w[k] & 0xFFFF0000u);
+                    } else {
+                        lo = __half2float(__ushort_as_half(uint16_t(w[k] & 0xFFFF)));
+                        hi = __half2float(__ushort_as_half(uint16_t(w[k] >> 16)));
+                    }
+                    sum += lo + hi;
+                }
+            }
+        }
+        acc = CarryT(sum);
+    }
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        CarryT tot = CarryT(0);
+        for (int k = 0; k < 8; ++k) tot += part[k];
+        reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(ws) + kHeaderBytes)[2 * size_t(t) + 1] = CO::enc(tot);
+    }
+}
+
+template <bool IS_INT>
+__global__ void __launch_bounds__(1024) tcu_totals_scan_kernel(void *ws, uint32_t tiles) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    __shared__ CarryT warp_part[32];
+    __shared__ CarryT running;
+    WsHeader *hdr = reinterpret_cast<WsHeader *>(ws);
+    uint64_t *rec = reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(ws) + kHeaderBytes);
+    const uint64_t flag = (uint64_t(hdr->epoch + 1) << 2) | kStatusInclusive;   // the epoch the main kernel will use
+    const uint32_t per = (tiles + 1023) / 1024;
+    const uint32_t lo = threadIdx.x * per, hi = min(lo + per, tiles);
+    CarryT mine = CarryT(0);
+    for (uint32_t i = lo; i < hi; ++i) mine += CO::dec(rec[2 * size_t(i) + 1]);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    CarryT inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        CarryT up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+    }
+    if (lane == 31) warp_part[wid] = inc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        CarryT r = CarryT(0);
+        for (int k = 0; k < 32; ++k) {
+            CarryT v = warp_part[k];
+            warp_part[k] = r;
+            r += v;
+        }
+        running = r;
+    }
+    __syncthreads();
+    CarryT acc = warp_part[wid] + (inc - mine);        // sum of everything before this thread's run
+    for (uint32_t i = lo; i < hi; ++i) {
+        acc += CO::dec(rec[2 * size_t(i) + 1]);
+        rec[2 * size_t(i) + 1] = CO::enc(acc);
+        rec[2 * size_t(i)] = flag;
     }
 }
 

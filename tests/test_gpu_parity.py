@@ -135,3 +135,25 @@ def test_stats_report(runner):
     assert st["tiles"] == n // TILE and st["s"] == 64 and st["sxs_products"] == n // (64 * 64)
     assert st["depth_bound"] == 2 * 3 and st["levels_used"] == 5 and st["variant"] == 0 and st["upper_level_path"] == 0
     assert st["mma_instructions"] == st["tiles"] * (2 * 4 + 8)      # U_64 products + row-total products
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f16", "bf16"])
+def test_two_sweep_variant_matches_oracle(runner, dtype):
+    # the reduce-then-scan structure (input read twice) must satisfy the same parity bars
+    from paper_2411_17887_b200 import binding as B
+    from tests.gpu_util import to_device, assert_int_equal, assert_float_close
+    for n, s in [(TILE, 16), (37 * TILE + 128 * 5 + 9, 64), (1500 * TILE + 77, 16)]:
+        x = gen(dtype, n, 4000 + n % 911)
+        d_in = to_device(x, dtype)
+        out = torch.empty(n, dtype=torch.int32 if dtype == "i8" else torch.float32, device="cuda")
+        B.check(B.tcu_scan_inclusive_twosweep(d_in, out, n, B.DTYPES[dtype], s, runner.ws_ptr, runner.ws_bytes, 0))
+        B.check(B.tcu_scan_device_status(runner.ws_ptr, 0))
+        assert B.tcu_scan_last_stats()["variant"] == 1
+        got = out.cpu().numpy()
+        if dtype == "i8":
+            assert_int_equal(got, x, False)
+        else:
+            assert_float_close(got, x, dtype, False)
+    # and the single-pass path still works on the same workspace afterwards
+    from tests.gpu_util import check
+    check(runner, gen(dtype, 5 * TILE + 3, 17), dtype, 16)
