@@ -291,6 +291,28 @@ def run_ours(args):
                 extras.append(time_extra(B, torch, "fp16 n=2^28 in the two-sweep structure, s=16",
                                          xf, 1, 1 << 28, 1, 16, False, ws_ptr, ws_bytes, two_sweep=True))
                 line["extra"] = extras
+            if args.sweep_ctas:
+                sms = torch.cuda.get_device_properties(local).multi_processor_count
+                sweep = []
+                ps = [1, 2, 4, 8, 16, 32, 64, 128, sms]
+                for pcount in ps:
+                    B.check(B.tcu_scan_set_max_ctas(pcount))
+                    reps = 2 if pcount < 8 else 5
+                    step()
+                    torch.cuda.synchronize()
+                    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a0.record()
+                    for _ in range(reps):
+                        step()
+                    a1.record()
+                    torch.cuda.synchronize()
+                    sweep.append({"p": pcount, "ms": a0.elapsed_time(a1) / reps})
+                B.check(B.tcu_scan_set_max_ctas(0))
+                t1 = sweep[0]["ms"]
+                for e in sweep:
+                    e["speedup_vs_p1"] = t1 / e["ms"]
+                    e["efficiency"] = t1 / e["ms"] / e["p"]
+                line["p_tcu_sweep"] = sweep
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -303,6 +325,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the timings of the other configurations")
+    ap.add_argument("--sweep-ctas", action="store_true",
+                    help="also time the headline scan on p = 1, 2, 4, ... persistent CTAs (one per SM) and report time vs p")
     ap.add_argument("--n-log2", type=int, default=28, help="log2 of the array length (28 = the headline workload)")
     ap.add_argument("--profile", action="store_true",
                     help="device-resident loop only (no end-to-end leg, no oracle): the command to wrap in ncu")

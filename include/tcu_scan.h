@@ -135,7 +135,8 @@ tcu_status_t tcu_scan_inclusive_twosweep(const void *d_in, void *d_out, size_t n
 
 /* `rows` independent scans of `cols` elements each, dense row-major (row stride = cols)
  * (Section 2.2 step 1: the algorithm run on each contiguous segment, no stitching).
- * cols must be a multiple of 128, else TCU_ERR_UNSUPPORTED.
+ * cols must be a multiple of 16 (so that every row starts 16-byte aligned in both arrays), else
+ * TCU_ERR_UNSUPPORTED.
  *   d_ws   at least tcu_scan_workspace_bytes(rows, cols, dt, s) bytes */
 tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols,
                               tcu_dtype_t dt, int s, int exclusive,
@@ -164,6 +165,12 @@ tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream);
  * stream has drained, tcu_scan_device_status(d_ws) returns TCU_ERR_TIMEOUT and the context is
  * still usable; tcu_scan_workspace_init() clears the condition.  Nothing faults or hangs. */
 tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned limit_ms, cudaStream_t stream);
+
+/* Experiment knob: run the following scans of this process on at most `max_ctas` persistent CTAs,
+ * i.e. on that many SMs (0 restores the default, one CTA per SM).  One CTA owns one SM's tensor
+ * core, so this is the p of the paper's p-TCU time bound O(n(1 + l/s^2)/p + (s^2 + l) log_s n)
+ * (Section 2.2, last paragraph, and the abstract).  Results do not depend on it. */
+tcu_status_t tcu_scan_set_max_ctas(int max_ctas);
 
 /* Copies the bookkeeping of the most recent scan call made by this process. */
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out);

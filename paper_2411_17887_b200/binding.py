@@ -52,6 +52,8 @@ _lib.tcu_scan_device_status.argtypes = [_vp, _vp]
 _lib.tcu_scan_device_status.restype = _int
 _lib.tcu_scan_selftest_timeout.argtypes = [_vp, _sz, ctypes.c_uint, _vp]
 _lib.tcu_scan_selftest_timeout.restype = _int
+_lib.tcu_scan_set_max_ctas.argtypes = [_int]
+_lib.tcu_scan_set_max_ctas.restype = _int
 _lib.tcu_scan_last_stats.argtypes = [ctypes.POINTER(TcuScanStats)]
 _lib.tcu_scan_last_stats.restype = _int
 _lib.tcu_status_string.argtypes = [_int]
@@ -118,6 +120,10 @@ def tcu_scan_device_status(d_ws, stream=0) -> int:
 
 def tcu_scan_selftest_timeout(d_ws, ws_bytes: int, limit_ms: int, stream=0) -> int:
     return _lib.tcu_scan_selftest_timeout(_p(d_ws), ws_bytes, int(limit_ms), stream)
+
+
+def tcu_scan_set_max_ctas(max_ctas: int) -> int:
+    return _lib.tcu_scan_set_max_ctas(int(max_ctas))
 
 
 def tcu_scan_last_stats() -> dict:

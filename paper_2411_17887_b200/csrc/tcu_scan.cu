@@ -32,6 +32,7 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+std::atomic<int> g_max_ctas{0};   // 0 = one CTA per SM; otherwise the persistent grid is capped (scaling experiments)
 std::mutex g_stats_mutex;
 tcu_scan_stats_t g_stats;
 bool g_have_stats = false;
@@ -109,7 +110,8 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     if (!d_in || !d_out) return TCU_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(d_in) & 15) || (reinterpret_cast<uintptr_t>(d_out) & 15)) return TCU_ERR_INVALID_ARG;
     const int eb = elem_bytes(dt);
-    if (rows > 1 && (cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
+    // batched rows: the row pitch must keep every row 16-byte aligned on both sides (TMA boxes, vector stores)
+    if (rows > 1 && ((cols * eb) % 16 != 0 || (cols * 4) % 16 != 0)) return TCU_ERR_UNSUPPORTED;
     if (level0 && (cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
     if (rows > (1ull << 31) || cols > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
     const uint64_t total = uint64_t(rows) * cols;
@@ -212,7 +214,10 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         }
         // persistent grid: every CTA must be resident at once (the carry chain waits on
         // lower-numbered tiles), so never more CTAs than SMs; one CTA fills an SM's shared memory
-        dim3 grid(unsigned(tiles < uint64_t(sms) ? tiles : uint64_t(sms)));
+        uint64_t ctas = uint64_t(sms);
+        const int cap = g_max_ctas.load();
+        if (cap > 0 && uint64_t(cap) < ctas) ctas = uint64_t(cap);
+        dim3 grid(unsigned(tiles < ctas ? tiles : ctas));
         st.grid = grid.x;
         cudaError_t e;
         if (dt == TCU_I8_I32)
@@ -221,14 +226,14 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
             e = exclusive ? dispatch_s<false, true>(s, prm, grid, smem, stream) : dispatch_s<false, false>(s, prm, grid, smem, stream);
         if (e != cudaSuccess) return TCU_ERR_CUDA;
     }
-    if (tail > 0) {   // only reachable with rows == 1
+    if (tail > 0) {   // the last cols % 128 elements of every scan
         const size_t start = size_t(rows128) * kTileCols;
         if (dt == TCU_I8_I32) {
-            if (exclusive) tcu_scan_tail_kernel<true, true><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
-            else tcu_scan_tail_kernel<true, false><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
+            if (exclusive) tcu_scan_tail_kernel<true, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
+            else tcu_scan_tail_kernel<true, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
         } else {
-            if (exclusive) tcu_scan_tail_kernel<false, true><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
-            else tcu_scan_tail_kernel<false, false><<<1, 128, 0, stream>>>(d_in, d_out, start, tail, d_ws, uint32_t(tiles), dt);
+            if (exclusive) tcu_scan_tail_kernel<false, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
+            else tcu_scan_tail_kernel<false, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
         }
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
     }
@@ -346,6 +351,12 @@ tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned lim
     if (limit_ms == 0 || limit_ms > 1000) return TCU_ERR_INVALID_ARG;
     tcu_scan_timeout_selftest_kernel<<<1, 32, 0, stream>>>(d_ws, (long long)limit_ms * 2000000LL);
     return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+}
+
+tcu_status_t tcu_scan_set_max_ctas(int max_ctas) {
+    if (max_ctas < 0) return TCU_ERR_INVALID_ARG;
+    g_max_ctas.store(max_ctas);
+    return TCU_OK;
 }
 
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out) {

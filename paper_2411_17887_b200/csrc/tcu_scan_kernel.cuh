@@ -422,7 +422,11 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     const uint32_t num_in = p.in_stages;
 
     // ---- set-up
-    if (threadIdx.x == 0) {
+    uint32_t first_ticket = 0;                 // (thread 0 only) claimed before anything else, so that the round trip
+    if (threadIdx.x == 0) {                    // of the atomic and of the epoch read overlap the rest of the set-up
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&p.tmap_in)) : "memory");
+        first_ticket = TCU_STATIC_TILES ? blockIdx.x : atomicAdd(&hdr->ticket, 1u);
+        const uint32_t prev_epoch = ld_relaxed_u32(&hdr->epoch);
         for (int i = 0; i < kMaxInStages; ++i) {
             mbar_init(smem_u32(&ctl->full[i]), 1);
             mbar_init(smem_u32(&ctl->empty[i]), 2);
@@ -441,7 +445,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
         }
         ctl->abort_flag = 0;
-        ctl->epoch = ld_relaxed_u32(&hdr->epoch) + 1;
+        ctl->epoch = prev_epoch + 1;
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -595,7 +599,10 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
                 PROF_ADD(0);
                 uint32_t t = kNoTile;
-                if (markers == 0) t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
+                if (markers == 0) {
+                    if (j == 0) t = first_ticket;
+                    else t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
+                }
                 if (t >= p.tiles_total) t = kNoTile;
                 PROF_ADD(1);
                 PROF_INC(3, 1);
@@ -923,14 +930,17 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 // Runs after the main kernel on the same stream; the carry is the inclusive record of the
 // last tile (or nothing when there is no full row).
 template <bool IS_INT, bool EXCL>
-__global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start, uint32_t count, const void *ws,
-                                     uint32_t tiles, uint32_t dtype) {
+__global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start0, size_t pitch, uint32_t count, const void *ws,
+                                     uint32_t tiles_per_row, uint32_t dtype) {
+    // one block per scan (blockIdx.x = row of a batched scan)
+    const size_t start = start0 + size_t(blockIdx.x) * pitch;
+    const uint32_t tiles = (blockIdx.x + 1) * tiles_per_row;      // index + 1 of this scan's last tile record
     using CO = CarryOps<IS_INT>;
     using CarryT = typename CO::T;
     __shared__ CarryT warp_tot[4];
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
     CarryT carry = CarryT(0);
-    if (tiles > 0) {
+    if (tiles_per_row > 0) {
         uint64_t flag, val;
         ld_record(reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes + size_t(tiles - 1) * 16, flag, val);
         carry = CO::dec(val);

@@ -110,7 +110,8 @@ def test_int_wraps_modulo_2_32(runner):
 @pytest.mark.parametrize("dtype", ["i8", "bf16", "f16"])
 def test_batched_rows(runner, dtype):
     from tests.gpu_util import check
-    for rows, cols in [(1, 128), (3, 128), (5, TILE), (4, 2 * TILE + 128 * 5), (64, 65536), (7, 128 * 129)]:
+    for rows, cols in [(1, 128), (3, 128), (5, TILE), (4, 2 * TILE + 128 * 5), (64, 65536), (7, 128 * 129),
+                       (6, 16), (9, 112), (5, 128 + 16), (3, TILE + 128 * 3 + 48), (33, 2 * TILE - 16)]:
         for s in (16, 128):
             check(runner, gen(dtype, (rows, cols), rows * 7 + cols % 101), dtype, s, False)
         check(runner, gen(dtype, (rows, cols), rows * 7 + cols % 103), dtype, 64, True)
@@ -157,3 +158,18 @@ def test_two_sweep_variant_matches_oracle(runner, dtype):
     # and the single-pass path still works on the same workspace afterwards
     from tests.gpu_util import check
     check(runner, gen(dtype, 5 * TILE + 3, 17), dtype, 16)
+
+
+def test_result_does_not_depend_on_the_number_of_ctas(runner):
+    # the p of the paper's p-TCU bound: any number of persistent CTAs gives the same integers
+    from paper_2411_17887_b200 import binding as B
+    from tests.gpu_util import check
+    x = gen("i8", 200 * TILE + 128 * 7 + 3, 99)
+    try:
+        for p in (1, 3, 32):
+            B.check(B.tcu_scan_set_max_ctas(p))
+            check(runner, x, "i8", 16)
+            assert B.tcu_scan_last_stats()["grid"] == p
+    finally:
+        B.check(B.tcu_scan_set_max_ctas(0))
+    assert B.tcu_scan_set_max_ctas(-1) == B.TCU_ERR_INVALID_ARG

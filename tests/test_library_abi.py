@@ -66,7 +66,7 @@ def test_argument_checks_return_before_any_launch(B):
     assert B.tcu_scan_exclusive(ok_in, ok_out, 10, 0, 16, None, 0) == B.TCU_ERR_WORKSPACE
     assert B.tcu_scan_exclusive(ok_in, ok_out, 1 << 20, 0, 16, ok_ws, 64) == B.TCU_ERR_WORKSPACE    # too small
     assert B.tcu_scan_inclusive(ok_in, ok_in + 64, 1 << 10, 0, 16, ok_ws, ws) == B.TCU_ERR_INVALID_ARG  # overlap
-    assert B.tcu_scan_batched(ok_in, ok_out, 4, 100, 0, 16, 0, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED  # cols % 128
+    assert B.tcu_scan_batched(ok_in, ok_out, 4, 100, 0, 16, 0, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED  # cols % 16
     assert B.tcu_scan_level0_debug(ok_in, ok_out, 100, 0, 16, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED
     assert B.tcu_scan_workspace_init(None, 1024, 0) == B.TCU_ERR_WORKSPACE
     assert B.tcu_scan_device_status(None, 0) == B.TCU_ERR_WORKSPACE
