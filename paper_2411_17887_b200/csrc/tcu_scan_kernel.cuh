@@ -26,23 +26,33 @@
 
 namespace tcu {
 
+// ---- compile-time knobs (the defaults are the measured best; the others exist for A/B builds)
 #ifndef TCU_STORE_GROUPS
-#define TCU_STORE_GROUPS 2
+#define TCU_STORE_GROUPS 2      // groups of four store warps (2 or 3)
 #endif
 #ifndef TCU_PREFETCH_DIST
-#define TCU_PREFETCH_DIST 256
+#define TCU_PREFETCH_DIST 256   // tiles ahead of the claimed one that are prefetched into L2 (0 = off)
 #endif
 #ifndef TCU_TMA_STORE
-#define TCU_TMA_STORE 0
+#define TCU_TMA_STORE 0         // 1 = write the output with TMA stores instead of st.global
+#endif
+#ifndef TCU_SLABS
+#define TCU_SLABS 2             // staging slabs per store warp in the TMA-store build
 #endif
 #ifndef TCU_SETMAXNREG
-#define TCU_SETMAXNREG 1
+#define TCU_SETMAXNREG 1        // move registers from the control warps to the store warps
 #endif
 #ifndef TCU_LOOKBACK
-#define TCU_LOOKBACK 2
+#define TCU_LOOKBACK 2          // windows of 32 records fetched per look-back round
 #endif
 #ifndef TCU_STATIC_TILES
-#define TCU_STATIC_TILES 0
+#define TCU_STATIC_TILES 0      // 1 = tile j of CTA b is b + j * gridDim.x instead of the next ticket
+#endif
+#ifndef TCU_MAX_STAGES
+#define TCU_MAX_STAGES 10       // most input stages the host will ask for
+#endif
+#ifndef TCU_PIPE_STORE
+#define TCU_PIPE_STORE 0        // 1 = fetch the next 32 TMEM columns before the current ones are stored
 #endif
 
 constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM lanes
@@ -53,11 +63,8 @@ constexpr int kNumTot = 8;              // TMEM accumulators of the row totals (
 constexpr int kTotCols = 16;
 constexpr int kTotBase = kNumAcc * kTileCols;            // first TMEM column of the totals ring
 static_assert(kTotBase + kNumTot * kTotCols <= 512, "TMEM has 512 columns");
-constexpr int kStoreGroups = TCU_STORE_GROUPS;           // groups of 4 store warps; group g takes the tiles with j % kStoreGroups == g
+constexpr int kStoreGroups = TCU_STORE_GROUPS;           // group g takes the tiles with j % kStoreGroups == g
 constexpr int kSlabBytes = 32 * 4 * 32;                  // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
-#ifndef TCU_SLABS
-#define TCU_SLABS 2
-#endif
 constexpr int kSlabsPerWarp = TCU_TMA_STORE ? TCU_SLABS : 1;   // TMA stores read the slab asynchronously: ring of slabs
 constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabsPerWarp * kSlabBytes;   // staging slabs of the store warps
 constexpr int kNumCarry = 16;           // tiles a CTA may have between "row totals known" and "stored": ring of carry entries
@@ -65,16 +72,10 @@ constexpr int kTileRing = 32;           // ring of claimed tile numbers (must ex
 constexpr uint32_t kNoTile = 0xFFFFFFFFu;   // "no more tiles" marker pushed through the pipeline
 constexpr int kNumLookbackWarps = 5;
 constexpr int kNumMarkers = kNumLookbackWarps;   // markers pushed: one per look-back warp
-#ifndef TCU_MAX_STAGES
-#define TCU_MAX_STAGES 10
-#endif
-#ifndef TCU_PIPE_STORE
-#define TCU_PIPE_STORE 0
-#endif
 constexpr int kMaxInStages = 12;        // size of the barrier arrays
-constexpr int kUseInStages = TCU_MAX_STAGES;   // most stages the host will ask for
-constexpr uint32_t kPrefetchDist = TCU_PREFETCH_DIST;   // tiles ahead of the claimed one that are prefetched into L2
-constexpr int kLookBack = TCU_LOOKBACK; // records fetched per lane and round of the cross-tile look-back
+constexpr int kUseInStages = TCU_MAX_STAGES;
+constexpr uint32_t kPrefetchDist = TCU_PREFETCH_DIST;
+constexpr int kLookBack = TCU_LOOKBACK;
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
 constexpr int kEpilogueThreads = 128;
@@ -85,8 +86,8 @@ constexpr int kStoreRegs = (kStoreGroups == 3) ? 104 : 128;
 static_assert(128 * (64 + 64 + 40 + kStoreGroups * kStoreRegs) <= 61440, "register pool");
 constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
-constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back
-constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps - 1);   // warp 3 is the first look-back warp
+constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back (warp 3 is one more)
+constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps - 1);
 
 // workspace: 256-byte header, then one 16-byte record per tile
 constexpr int kHeaderBytes = 256;
