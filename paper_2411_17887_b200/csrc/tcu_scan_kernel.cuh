@@ -22,6 +22,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 namespace tcu {
@@ -424,30 +425,33 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 
     // ---- set-up
     uint32_t first_ticket = 0;                 // (thread 0 only) claimed before anything else, so that the round trip
-    if (threadIdx.x == 0) {                    // of the atomic and of the epoch read overlap the rest of the set-up
+    uint32_t prev_epoch = 0;                   // of the atomic and of the epoch read overlap the rest of the set-up
+    if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&p.tmap_in)) : "memory");
         first_ticket = TCU_STATIC_TILES ? blockIdx.x : atomicAdd(&hdr->ticket, 1u);
-        const uint32_t prev_epoch = ld_relaxed_u32(&hdr->epoch);
-        for (int i = 0; i < kMaxInStages; ++i) {
-            mbar_init(smem_u32(&ctl->full[i]), 1);
-            mbar_init(smem_u32(&ctl->empty[i]), 2);
+        prev_epoch = ld_relaxed_u32(&hdr->epoch);
+    }
+    {
+        // the barriers are the first kNumBarriers 64-bit words of the control block: one thread each
+        constexpr int kNumBarriers = 2 * kMaxInStages + 2 * kNumAcc + 2 * kNumTot + 3 * kNumCarry;
+        static_assert(kNumBarriers <= kThreads, "one thread per barrier");
+        static_assert(offsetof(SmemCtl, agg_slot) == kNumBarriers * 8, "barriers must be contiguous");
+        const int k = threadIdx.x;
+        if (k < kNumBarriers) {
+            uint32_t count = 1;                                                 // full, acc_full, tot_full, carry_ready
+            if (k >= kMaxInStages && k < 2 * kMaxInStages) count = 2;           // empty: both MMA issuers
+            const int kAccEmpty = 2 * kMaxInStages + kNumAcc, kTotEmpty = kAccEmpty + kNumAcc + kNumTot;
+            const int kRingFree = kTotEmpty + kNumTot, kCarryReady = kRingFree + 2 * kNumCarry;
+            if (k >= kAccEmpty && k < kAccEmpty + kNumAcc) count = kEpilogueThreads;        // acc_empty
+            if (k >= kTotEmpty && k < kTotEmpty + kNumTot) count = kEpilogueThreads;        // tot_empty
+            if (k >= kRingFree && k < kCarryReady) count = kEpilogueThreads;                // ring_free, agg_ready
+            mbar_init(smem_u32(reinterpret_cast<uint64_t *>(ctl) + k), count);
+            fence_barrier_init();
         }
-        for (int i = 0; i < kNumAcc; ++i) {
-            mbar_init(smem_u32(&ctl->acc_full[i]), 1);
-            mbar_init(smem_u32(&ctl->acc_empty[i]), kEpilogueThreads);
-        }
-        for (int i = 0; i < kNumTot; ++i) {
-            mbar_init(smem_u32(&ctl->tot_full[i]), 1);
-            mbar_init(smem_u32(&ctl->tot_empty[i]), kEpilogueThreads);
-        }
-        for (int i = 0; i < kNumCarry; ++i) {
-            mbar_init(smem_u32(&ctl->ring_free[i]), kEpilogueThreads);
-            mbar_init(smem_u32(&ctl->agg_ready[i]), kEpilogueThreads);
-            mbar_init(smem_u32(&ctl->carry_ready[i]), 1);
-        }
+    }
+    if (threadIdx.x == 0) {
         ctl->abort_flag = 0;
         ctl->epoch = prev_epoch + 1;
-        fence_barrier_init();
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), 512);
