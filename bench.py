@@ -30,9 +30,9 @@ N_ELEMS = 1 << 28
 S_TILE = 16
 BYTES_PER_ELEM = 5          # int8 read + int32 written
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel, from the ncu
-# capture summarised in profiles/ (scaled to a full launch as described there); None until captured
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 4 * 277.15e6   # profiles/tcu_scan_kernel_int8_s16_n2p26_ncu_full.md, scaled x4 to n = 2^28
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel on 2^26 elements, from the
+# ncu capture summarised in profiles/ (traffic grows in proportion to n: one read and one write per element)
+NCU_TRAFFIC_BYTES_PER_2P26 = 277.15e6   # profiles/tcu_scan_kernel_int8_s16_n2p26_ncu_full.md; scaled by n / 2^26 below
 
 
 def measured_peak():
@@ -255,7 +255,7 @@ def run_ours(args):
                        "hbm_gb_per_s": achieved, "pct_of_8TBps": 100 * achieved / 8000.0,
                        "pct_of_measured_copy": 100 * achieved / peak},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": f"of {peak_kind}",
+                         "traffic": NCU_TRAFFIC_BYTES_PER_2P26 * n / (1 << 26), "peak_kind": f"of {peak_kind}",
                          "kernel": "tcu_scan_kernel<int8,s=16,inclusive>", "algorithmic_bytes_per_launch": BYTES_PER_ELEM * n},
             "e2e": {"value": world * n * e2e_steps / e2e_s, "unit": "elements/s", "h2d_bytes_per_step": n,
                     "d2h_bytes_per_step": 4 * n, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps},

@@ -73,3 +73,17 @@ def test_batched_config_C4(runner):
         y, a = so.scan_f64(so.widen(xs, cfg.dtype))
         err = np.abs(got[r0:r0 + block].astype(np.float64) - y)
         assert (err <= so.float_tolerance(a)).all(), f"rows {r0}.."
+
+
+def test_beyond_four_gigabytes_of_output():
+    # n = 2^30 + 12345 int8: the output is larger than 4 GiB, so every 32-bit index or byte offset would show
+    from tests.gpu_util import Runner
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    n = (1 << 30) + 12345
+    x = inputs.int8_uniform(n, -127, 127, 31)
+    big = Runner(1, n)
+    got = big.run(x, "i8", 16)
+    compare_piecewise(got, x, "i8", False)
+    got = big.run(x, "i8", 128, exclusive=True)
+    compare_piecewise(got, x, "i8", True)
