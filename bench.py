@@ -290,6 +290,26 @@ def run_ours(args):
                                          d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes, two_sweep=True))
                 extras.append(time_extra(B, torch, "fp16 n=2^28 in the two-sweep structure, s=16",
                                          xf, 1, 1 << 28, 1, 16, False, ws_ptr, ws_bytes, two_sweep=True))
+                # application: radix sort of 2^24 keys by 32 one-bit splits, each an exclusive scan of int8 flags
+                ns = 1 << 24
+                keys = torch.randint(0, 1 << 31, (ns,), device="cuda", dtype=torch.int32, generator=g)
+                sorted_out = torch.empty_like(keys)
+                tmp_bytes = B.tcu_sort_tmp_bytes(ns)
+                tmp = torch.empty(tmp_bytes + 256, dtype=torch.uint8, device="cuda")
+                tmp_ptr = tmp.data_ptr() + (-tmp.data_ptr()) % 256
+                for _ in range(2):
+                    B.check(B.tcu_sort_u32(keys, sorted_out, ns, tmp_ptr, tmp_bytes, ws_ptr, ws_bytes, stream))
+                torch.cuda.synchronize()
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0.record()
+                for _ in range(3):
+                    B.check(B.tcu_sort_u32(keys, sorted_out, ns, tmp_ptr, tmp_bytes, ws_ptr, ws_bytes, stream))
+                s1.record()
+                torch.cuda.synchronize()
+                ms_sort = s0.elapsed_time(s1) / 3
+                ok = bool((sorted_out[1:] >= sorted_out[:-1]).all())
+                extras.append({"workload": "radix sort of 2^24 uint32 keys by 32 one-bit splits (32 exclusive scans)",
+                               "ms": ms_sort, "keys_per_s": ns / (ms_sort * 1e-3), "sorted": ok})
                 line["extra"] = extras
             if args.sweep_ctas:
                 sms = torch.cuda.get_device_properties(local).multi_processor_count

@@ -166,6 +166,18 @@ tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream);
  * still usable; tcu_scan_workspace_init() clears the condition.  Nothing faults or hangs. */
 tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned limit_ms, cudaStream_t stream);
 
+/* Radix sort of 32-bit unsigned keys by 32 stable one-bit splits, each split an exclusive
+ * tcu scan of int8 flags (the paper's introduction: with Blelloch's reduction of radix sort to
+ * prefix sums, a tensor-core-unit machine can sort).  An application of the scan, not a tuned
+ * sort.
+ *   d_keys_in / d_keys_out   device, n keys each, 16-byte aligned, must not overlap
+ *   d_tmp                    device scratch of tcu_sort_tmp_bytes(n) bytes, 256-byte aligned
+ *   d_ws                     scan workspace of tcu_scan_workspace_bytes(1, n, TCU_I8_I32, 16) bytes
+ *   n < 2^31 */
+size_t tcu_sort_tmp_bytes(size_t n);
+tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_t n, void *d_tmp, size_t tmp_bytes,
+                          void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
 /* Experiment knob: run the following scans of this process on at most `max_ctas` persistent CTAs,
  * i.e. on that many SMs (0 restores the default, one CTA per SM).  One CTA owns one SM's tensor
  * core, so this is the p of the paper's p-TCU time bound O(n(1 + l/s^2)/p + (s^2 + l) log_s n)

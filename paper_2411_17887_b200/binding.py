@@ -52,6 +52,10 @@ _lib.tcu_scan_device_status.argtypes = [_vp, _vp]
 _lib.tcu_scan_device_status.restype = _int
 _lib.tcu_scan_selftest_timeout.argtypes = [_vp, _sz, ctypes.c_uint, _vp]
 _lib.tcu_scan_selftest_timeout.restype = _int
+_lib.tcu_sort_tmp_bytes.argtypes = [_sz]
+_lib.tcu_sort_tmp_bytes.restype = _sz
+_lib.tcu_sort_u32.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _sz, _vp]
+_lib.tcu_sort_u32.restype = _int
 _lib.tcu_scan_set_max_ctas.argtypes = [_int]
 _lib.tcu_scan_set_max_ctas.restype = _int
 _lib.tcu_scan_last_stats.argtypes = [ctypes.POINTER(TcuScanStats)]
@@ -120,6 +124,14 @@ def tcu_scan_device_status(d_ws, stream=0) -> int:
 
 def tcu_scan_selftest_timeout(d_ws, ws_bytes: int, limit_ms: int, stream=0) -> int:
     return _lib.tcu_scan_selftest_timeout(_p(d_ws), ws_bytes, int(limit_ms), stream)
+
+
+def tcu_sort_tmp_bytes(n: int) -> int:
+    return int(_lib.tcu_sort_tmp_bytes(n))
+
+
+def tcu_sort_u32(d_keys_in, d_keys_out, n: int, d_tmp, tmp_bytes: int, d_ws, ws_bytes: int, stream=0) -> int:
+    return _lib.tcu_sort_u32(_p(d_keys_in), _p(d_keys_out), n, _p(d_tmp), tmp_bytes, _p(d_ws), ws_bytes, stream)
 
 
 def tcu_scan_set_max_ctas(max_ctas: int) -> int:

@@ -10,6 +10,7 @@
 #include <mutex>
 
 #include "tcu_scan_kernel.cuh"
+#include "tcu_split.cuh"
 
 namespace {
 
@@ -351,6 +352,40 @@ tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned lim
     if (limit_ms == 0 || limit_ms > 1000) return TCU_ERR_INVALID_ARG;
     tcu_scan_timeout_selftest_kernel<<<1, 32, 0, stream>>>(d_ws, (long long)limit_ms * 2000000LL);
     return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+}
+
+size_t tcu_sort_tmp_bytes(size_t n) {
+    // flags (n bytes, padded), scanned flags (4 n), second key buffer (4 n); each part 256-byte aligned
+    const size_t a = (n + 255) & ~size_t(255), b = (4 * n + 255) & ~size_t(255);
+    return a + 2 * b + 256;
+}
+
+tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_t n, void *d_tmp, size_t tmp_bytes,
+                          void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    if (n == 0) return TCU_OK;
+    if (!d_keys_in || !d_keys_out || !d_tmp) return TCU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_keys_in) & 15) || (reinterpret_cast<uintptr_t>(d_keys_out) & 15) ||
+        (reinterpret_cast<uintptr_t>(d_tmp) & 255))
+        return TCU_ERR_INVALID_ARG;
+    if (n >= (size_t(1) << 31)) return TCU_ERR_UNSUPPORTED;          // positions are int32 scan results
+    if (tmp_bytes < tcu_sort_tmp_bytes(n)) return TCU_ERR_WORKSPACE;
+    const size_t a = (n + 255) & ~size_t(255), b = (4 * n + 255) & ~size_t(255);
+    int8_t *flags = reinterpret_cast<int8_t *>(d_tmp);
+    int32_t *f = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(d_tmp) + a);
+    uint32_t *other = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_tmp) + a + b);
+    // 32 passes ping-pong between `other` and d_keys_out so that the last pass lands in d_keys_out
+    const uint32_t *src = d_keys_in;
+    for (int bit = 0; bit < 32; ++bit) {
+        uint32_t *dst = (bit & 1) ? d_keys_out : other;
+        const unsigned blocks4 = unsigned((n + 4 * 256 - 1) / (4 * 256));
+        split_flags_kernel<<<blocks4, 256, 0, stream>>>(src, flags, n, bit);
+        tcu_status_t st = scan_impl(flags, f, 1, n, TCU_I8_I32, 16, true, false, d_ws, ws_bytes, stream);
+        if (st != TCU_OK) return st;
+        split_scatter_kernel<<<unsigned((n + 255) / 256), 256, 0, stream>>>(src, flags, f, dst, n);
+        if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+        src = dst;
+    }
+    return TCU_OK;
 }
 
 tcu_status_t tcu_scan_set_max_ctas(int max_ctas) {
