@@ -148,10 +148,13 @@ tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t
 tcu_status_t tcu_scan_level0_debug(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                    void *d_ws, size_t ws_bytes, cudaStream_t stream);
 
-/* Host-buffer form: copies h_in to d_in (host->device), scans, copies d_out to h_out
- * (device->host), all asynchronously on `stream`; the caller synchronises the stream
- * before reading h_out.  h_in / h_out should be pinned for the copies to be asynchronous.
- * d_in / d_out are caller-owned device staging buffers of n input / n output elements. */
+/* Host-buffer form: uploads h_in to d_in, scans, downloads d_out to h_out.  Everything is
+ * asynchronous; the caller synchronises `stream` before reading h_out (that also covers the
+ * copies, which long inclusive scans run on two internal streams so that upload, scan and
+ * download of successive 2^24-element pieces overlap; each piece continues from the last output
+ * of the piece before it).  h_in / h_out should be pinned, otherwise the copies serialise.
+ * d_in / d_out are caller-owned device staging buffers of n input / n output elements; they and
+ * the workspace are in use until `stream` has drained. */
 tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t dt, int s, int exclusive,
                            void *d_in, void *d_out, void *d_ws, size_t ws_bytes, cudaStream_t stream);
 

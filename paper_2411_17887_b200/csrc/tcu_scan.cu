@@ -105,7 +105,7 @@ bool overlaps(const void *a, size_t an, const void *b, size_t bn) {
 
 tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
                        bool exclusive, bool level0, void *d_ws, size_t ws_bytes, cudaStream_t stream,
-                       bool two_sweep = false) {
+                       bool two_sweep = false, const void *d_carry_in = nullptr) {
     if (!valid_dtype(dt) || !valid_s(s)) return (s > 0 && valid_dtype(dt)) ? TCU_ERR_UNSUPPORTED : TCU_ERR_INVALID_ARG;
     if (rows == 0 || cols == 0) return TCU_OK;
     if (!d_in || !d_out) return TCU_ERR_INVALID_ARG;
@@ -192,6 +192,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         }
         prm.ws = d_ws;
         prm.out = d_out;
+        prm.carry_in = (rows == 1 && !two_sweep) ? d_carry_in : nullptr;
         prm.scan_pitch = cols;
         prm.rows128 = uint32_t(rows128);
         prm.tiles_total = uint32_t(tiles);
@@ -230,11 +231,11 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     if (tail > 0) {   // the last cols % 128 elements of every scan
         const size_t start = size_t(rows128) * kTileCols;
         if (dt == TCU_I8_I32) {
-            if (exclusive) tcu_scan_tail_kernel<true, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
-            else tcu_scan_tail_kernel<true, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
+            if (exclusive) tcu_scan_tail_kernel<true, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
+            else tcu_scan_tail_kernel<true, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
         } else {
-            if (exclusive) tcu_scan_tail_kernel<false, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
-            else tcu_scan_tail_kernel<false, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt);
+            if (exclusive) tcu_scan_tail_kernel<false, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
+            else tcu_scan_tail_kernel<false, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
         }
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
     }
@@ -269,6 +270,37 @@ tcu_status_t noalloc_scratch(void **out) {
     }
     *out = addr[dev];
     return TCU_OK;
+}
+
+// Streams and events of the pipelined host-buffer entry point: created on first use, per device, kept
+// for the life of the process (host-side objects; no device memory).
+struct HostPipe {
+    static constexpr int kEvents = 64;      // far more than the pieces that can be in flight at once
+    cudaStream_t up = nullptr, down = nullptr;
+    cudaEvent_t start = nullptr, finish = nullptr;
+    cudaEvent_t ev[kEvents] = {};
+    bool ok = false;
+};
+
+HostPipe *host_pipe() {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static HostPipe pipes[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    HostPipe &p = pipes[dev];
+    if (!p.ok) {
+        bool good = cudaStreamCreateWithFlags(&p.up, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&p.down, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&p.finish, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; good && i < HostPipe::kEvents; ++i)
+            good = cudaEventCreateWithFlags(&p.ev[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!good) return nullptr;
+        p.ok = true;
+    }
+    return &p;
 }
 
 }  // namespace
@@ -331,11 +363,41 @@ tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t 
     if (!valid_dtype(dt)) return TCU_ERR_INVALID_ARG;
     if (n == 0) return TCU_OK;
     if (!h_in || !h_out || !d_in || !d_out) return TCU_ERR_INVALID_ARG;
-    if (cudaMemcpyAsync(d_in, h_in, n * elem_bytes(dt), cudaMemcpyHostToDevice, stream) != cudaSuccess) return TCU_ERR_CUDA;
-    tcu_status_t st = scan_impl(d_in, d_out, 1, n, dt, s, exclusive != 0, false, d_ws, ws_bytes, stream);
-    if (st != TCU_OK) return st;
-    if (cudaMemcpyAsync(h_out, d_out, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TCU_ERR_CUDA;
-    return TCU_OK;
+    const size_t eb = size_t(elem_bytes(dt));
+    constexpr size_t kChunk = size_t(1) << 24;                 // elements per piece (a multiple of the tile)
+    HostPipe *pipe = (exclusive || n <= 2 * kChunk) ? nullptr : host_pipe();
+    if (!pipe) {                                               // short or exclusive: one copy in, one scan, one copy out
+        if (cudaMemcpyAsync(d_in, h_in, n * eb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return TCU_ERR_CUDA;
+        tcu_status_t st = scan_impl(d_in, d_out, 1, n, dt, s, exclusive != 0, false, d_ws, ws_bytes, stream);
+        if (st != TCU_OK) return st;
+        if (cudaMemcpyAsync(h_out, d_out, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TCU_ERR_CUDA;
+        return TCU_OK;
+    }
+    // Long inclusive scans are cut into pieces: the upload of piece i+1, the scan of piece i (continuing from the
+    // last output of piece i-1) and the download of piece i-1 overlap, each on its own stream.
+    const uint8_t *hi = reinterpret_cast<const uint8_t *>(h_in);
+    uint8_t *ho = reinterpret_cast<uint8_t *>(h_out);
+    uint8_t *di = reinterpret_cast<uint8_t *>(d_in), *dout = reinterpret_cast<uint8_t *>(d_out);
+    if (cudaEventRecord(pipe->start, stream) != cudaSuccess) return TCU_ERR_CUDA;    // the caller's earlier work comes first
+    cudaStreamWaitEvent(pipe->up, pipe->start, 0);
+    cudaStreamWaitEvent(pipe->down, pipe->start, 0);
+    const size_t pieces = (n + kChunk - 1) / kChunk;
+    for (size_t i = 0; i < pieces; ++i) {
+        const size_t lo = i * kChunk, len = (lo + kChunk <= n) ? kChunk : n - lo;
+        cudaEvent_t up_done = pipe->ev[(2 * i) % HostPipe::kEvents], scan_done = pipe->ev[(2 * i + 1) % HostPipe::kEvents];
+        if (cudaMemcpyAsync(di + lo * eb, hi + lo * eb, len * eb, cudaMemcpyHostToDevice, pipe->up) != cudaSuccess) return TCU_ERR_CUDA;
+        cudaEventRecord(up_done, pipe->up);
+        cudaStreamWaitEvent(stream, up_done, 0);
+        tcu_status_t st = scan_impl(di + lo * eb, dout + lo * 4, 1, len, dt, s, false, false, d_ws, ws_bytes, stream, false,
+                                    i == 0 ? nullptr : dout + (lo - 1) * 4);
+        if (st != TCU_OK) return st;
+        cudaEventRecord(scan_done, stream);
+        cudaStreamWaitEvent(pipe->down, scan_done, 0);
+        if (cudaMemcpyAsync(ho + lo * 4, dout + lo * 4, len * 4, cudaMemcpyDeviceToHost, pipe->down) != cudaSuccess) return TCU_ERR_CUDA;
+    }
+    if (cudaEventRecord(pipe->finish, pipe->down) != cudaSuccess) return TCU_ERR_CUDA;
+    cudaStreamWaitEvent(stream, pipe->finish, 0);              // synchronising `stream` now covers the downloads too
+    return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
 }
 
 tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream) {

@@ -136,6 +136,7 @@ struct alignas(64) ScanParams {
     CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 32 (used by the TMA-store variant)
     void *ws;
     void *out;                // output array (4-byte elements)
+    const void *carry_in;     // optional: one output-typed value added to every element of a single-array scan (or NULL)
     uint64_t scan_pitch;      // elements between consecutive scans (batched), unused for a single array
     uint32_t rows128;         // full 128-element rows of one scan
     uint32_t tiles_total;     // all tiles of the launch
@@ -164,6 +165,7 @@ struct SmemCtl {
     uint32_t tile_of[kTileRing];     // tile number of the j-th tile claimed by this CTA
     uint32_t tmem_base;
     uint32_t epoch;
+    uint32_t carry_in_bits;          // value at *carry_in (0 when there is none)
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 2048;
@@ -452,6 +454,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     if (threadIdx.x == 0) {
         ctl->abort_flag = 0;
         ctl->epoch = prev_epoch + 1;
+        ctl->carry_in_bits = p.carry_in ? *reinterpret_cast<const uint32_t *>(p.carry_in) : 0u;
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), 512);
@@ -487,6 +490,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 
     const uint32_t tmem_base = ctl->tmem_base;
     const uint32_t epoch = ctl->epoch;
+    // what precedes the whole scan (continuation of an earlier segment); only single-array calls pass one
+    const CarryT carry_in = IS_INT ? CarryT(ctl->carry_in_bits) : CarryT(__uint_as_float(ctl->carry_in_bits));
     Waiter w{ctl, hdr};
 
     // The j-th tile handled by this CTA is number tile_of[j % kTileRing]: either blockIdx.x + j * gridDim.x
@@ -512,7 +517,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (lane == 0) TRACE(t, 4);
             const CarryT agg = CO::dec(ctl->agg_slot[ts]);
             const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
-            CarryT prefix = CarryT(0);
+            CarryT prefix = (static_cast<int>(t) == t0) ? carry_in : CarryT(0);
             if (static_cast<int>(t) != t0) {       // (the first tile's record was published by the totals warps)
                 int pos = static_cast<int>(t) - 1;
                 bool gave_up = false;
@@ -785,8 +790,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
                 CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
                 // the first tile of a scan has nothing before it: its total is already inclusive
-                const uint32_t status = (t % p.tiles_per_row == 0) ? kStatusInclusive : kStatusPartial;
-                if (!p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(a));
+                const bool first = (t % p.tiles_per_row == 0);
+                const uint32_t status = first ? kStatusInclusive : kStatusPartial;
+                if (!p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
                 TRACE(t, 3);
                 ctl->agg_slot[ts] = CO::enc(a);
             }
@@ -936,7 +942,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 // last tile (or nothing when there is no full row).
 template <bool IS_INT, bool EXCL>
 __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start0, size_t pitch, uint32_t count, const void *ws,
-                                     uint32_t tiles_per_row, uint32_t dtype) {
+                                     uint32_t tiles_per_row, uint32_t dtype, const void *carry_in) {
     // one block per scan (blockIdx.x = row of a batched scan)
     const size_t start = start0 + size_t(blockIdx.x) * pitch;
     const uint32_t tiles = (blockIdx.x + 1) * tiles_per_row;      // index + 1 of this scan's last tile record
@@ -945,6 +951,10 @@ __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start0, s
     __shared__ CarryT warp_tot[4];
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
     CarryT carry = CarryT(0);
+    if (carry_in && tiles_per_row == 0) {       // no full row before the tail: the continuation value is all there is
+        const uint32_t bits = *reinterpret_cast<const uint32_t *>(carry_in);
+        carry = IS_INT ? CarryT(bits) : CarryT(__uint_as_float(bits));
+    }
     if (tiles_per_row > 0) {
         uint64_t flag, val;
         ld_record(reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes + size_t(tiles - 1) * 16, flag, val);
