@@ -74,8 +74,24 @@ cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStrea
         if (e != cudaSuccess) return e;
         configured.store(dev);
     }
+#if TCU_PDL
+    // programmatic dependent launch: this kernel's set-up (barriers, TMEM, constant operands) may overlap the
+    // tail of whatever runs before it in the stream; it waits (griddepcontrol.wait) before touching global memory
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tcu_scan_kernel<IS_INT, S, EXCL>, prm);
+#else
     tcu_scan_kernel<IS_INT, S, EXCL><<<grid, kThreads, smem, stream>>>(prm);
     return cudaGetLastError();
+#endif
 }
 
 template <bool IS_INT, bool EXCL>

@@ -34,6 +34,9 @@ namespace tcu {
 #ifndef TCU_PREFETCH_DIST
 #define TCU_PREFETCH_DIST 256   // tiles ahead of the claimed one that are prefetched into L2 (0 = off)
 #endif
+#ifndef TCU_PDL
+#define TCU_PDL 1               // programmatic dependent launch: set-up overlaps the tail of the previous kernel in the stream
+#endif
 #ifndef TCU_TMA_STORE
 #define TCU_TMA_STORE 0         // 1 = write the output with TMA stores instead of st.global
 #endif
@@ -119,7 +122,9 @@ __device__ __forceinline__ unsigned long long prof_now() {
 }
 #define TRACE(tile, k) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = prof_now(); } while (0)
 #define TRACE_V(tile, k, v) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = (v); } while (0)
+#define PROF_STAMP(k) do { if (g_prof && threadIdx.x == 0) g_prof[blockIdx.x * 64 + 48 + (k)] = prof_now(); } while (0)
 #else
+#define PROF_STAMP(k)
 #define TRACE(tile, k)
 #define TRACE_V(tile, k, v)
 #define PROF_DECL
@@ -166,6 +171,7 @@ struct SmemCtl {
     uint32_t tmem_base;
     uint32_t epoch;
     uint32_t carry_in_bits;          // value at *carry_in (0 when there is none)
+    uint64_t epoch_ready;            // thread 0 -> totals and look-back warps: epoch and carry_in_bits are written
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 2048;
@@ -426,12 +432,16 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     const uint32_t num_in = p.in_stages;
 
     // ---- set-up
+    PROF_STAMP(0);
     uint32_t first_ticket = 0;                 // (thread 0 only) claimed before anything else, so that the round trip
     uint32_t prev_epoch = 0;                   // of the atomic and of the epoch read overlap the rest of the set-up
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&p.tmap_in)) : "memory");
+#if !TCU_PDL
         first_ticket = TCU_STATIC_TILES ? blockIdx.x : atomicAdd(&hdr->ticket, 1u);
         prev_epoch = ld_relaxed_u32(&hdr->epoch);
+#endif
+        mbar_init(smem_u32(&ctl->epoch_ready), 1);
     }
     {
         // the barriers are the first kNumBarriers 64-bit words of the control block: one thread each
@@ -451,11 +461,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             fence_barrier_init();
         }
     }
-    if (threadIdx.x == 0) {
-        ctl->abort_flag = 0;
-        ctl->epoch = prev_epoch + 1;
-        ctl->carry_in_bits = p.carry_in ? *reinterpret_cast<const uint32_t *>(p.carry_in) : 0u;
-    }
+    if (threadIdx.x == 0) ctl->abort_flag = 0;
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), 512);
         tmem_relinquish();
@@ -488,11 +494,27 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
 
+    PROF_STAMP(1);
+    // Everything above touched only this CTA's shared memory and TMEM, so under programmatic dependent launch it
+    // may run while the previous kernel of the stream is still finishing.  From here on global memory is read.
+#if TCU_PDL
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
     const uint32_t tmem_base = ctl->tmem_base;
-    const uint32_t epoch = ctl->epoch;
-    // what precedes the whole scan (continuation of an earlier segment); only single-array calls pass one
-    const CarryT carry_in = IS_INT ? CarryT(ctl->carry_in_bits) : CarryT(__uint_as_float(ctl->carry_in_bits));
     Waiter w{ctl, hdr};
+    uint32_t my_epoch = 0;                     // (thread 0 only) the epoch of this launch
+    if (threadIdx.x == 0) {
+#if TCU_PDL
+        first_ticket = TCU_STATIC_TILES ? blockIdx.x : atomicAdd(&hdr->ticket, 1u);
+        prev_epoch = ld_relaxed_u32(&hdr->epoch);
+#endif
+        my_epoch = prev_epoch + 1;
+        ctl->epoch = my_epoch;
+        // what precedes the whole scan (continuation of an earlier segment); only single-array calls pass one
+        ctl->carry_in_bits = p.carry_in ? *reinterpret_cast<const uint32_t *>(p.carry_in) : 0u;
+        mbar_arrive(smem_u32(&ctl->epoch_ready));
+    }
 
     // The j-th tile handled by this CTA is number tile_of[j % kTileRing]: either blockIdx.x + j * gridDim.x
     // (static order) or the next ticket from the workspace (tiles claimed at run time, in increasing order:
@@ -501,6 +523,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     // that every role - and each of the look-back warps - sees one and stops.
     // ------------------------------------------------------------------ cross-tile carry scan (role of warp 3 and warps 20-23)
     auto lookback_role = [&](const uint32_t lbw) {
+        if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->epoch_ready), 0))) return;
+        const uint32_t epoch = ctl->epoch;
+        const CarryT carry_in = IS_INT ? CarryT(ctl->carry_in_bits) : CarryT(__uint_as_float(ctl->carry_in_bits));
         // ------------------------------------------------------------------ cross-tile carry scan
         // kNumLookbackWarps warps take the tiles in turn, so that the look-backs of the tiles in flight overlap.
         PROF_DECL
@@ -745,6 +770,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const int r = threadIdx.x - kFirstTotalsWarp * 32;          // tile row owned by this thread = TMEM lane
         const int wq = r >> 5;
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
+        const bool epoch_ok = w.wait(smem_u32(&ctl->epoch_ready), 0);
+        const uint32_t epoch = ctl->epoch;
+        const CarryT carry_in = IS_INT ? CarryT(ctl->carry_in_bits) : CarryT(__uint_as_float(ctl->carry_in_bits));
         uint32_t markers = 0;
         PROF_DECL
         PROF_T0();
@@ -752,7 +780,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             const uint32_t tt = j % kNumTot, utt = j / kNumTot;      // row-total accumulator in TMEM
             const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;   // carry ring entry
             // a wait that ran out is voted on, so that all 128 threads leave together
-            bool ok = w.wait(smem_u32(&ctl->tot_full[tt]), utt & 1);
+            bool ok = w.wait(smem_u32(&ctl->tot_full[tt]), utt & 1) && epoch_ok;
             ok = w.wait(smem_u32(&ctl->ring_free[ts]), (ut & 1) ^ 1) && ok;
             PROF_ADD(0);
             if (named_barrier_or(2, kEpilogueThreads, !ok)) break;
@@ -921,8 +949,10 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     }
 
     // ---- tear-down
+    PROF_STAMP(2);
     tc_fence_before();
     __syncthreads();
+    PROF_STAMP(3);
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0) {
@@ -932,9 +962,10 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             hdr->done = 0;
             hdr->ticket = 0;
             __threadfence();
-            hdr->epoch = epoch;
+            hdr->epoch = my_epoch;
         }
     }
+    PROF_STAMP(4);
 }
 
 // Tail of a single-array scan: the n % 128 elements after the last full 128-element row.
