@@ -290,6 +290,11 @@ def run_ours(args):
                                          d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes, two_sweep=True))
                 extras.append(time_extra(B, torch, "fp16 n=2^28 in the two-sweep structure, s=16",
                                          xf, 1, 1 << 28, 1, 16, False, ws_ptr, ws_bytes, two_sweep=True))
+                # the same scan with the row-total level on tensor cores (8-bit limbs) instead of warp shuffles
+                B.check(B.tcu_scan_set_upper_level_path(1))
+                extras.append(time_extra(B, torch, "C3 with the scan over row totals as a tcgen05 product on 8-bit limbs (upper_level_path = 1)",
+                                         d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes))
+                B.check(B.tcu_scan_set_upper_level_path(0))
                 # application: radix sort of 2^24 keys by 32 one-bit splits, each an exclusive scan of int8 flags
                 ns = 1 << 24
                 keys = torch.randint(0, 1 << 31, (ns,), device="cuda", dtype=torch.int32, generator=g)

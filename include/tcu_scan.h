@@ -64,7 +64,8 @@ typedef struct {
     uint64_t rows, cols;        /* problem shape (rows = 1 for the single-array calls)               */
     uint32_t s, dtype, exclusive;
     uint32_t variant;           /* 0 = single pass, decoupled look-back; 1 = two sweeps                 */
-    uint32_t upper_level_path;  /* 0 = levels above the U_s product run on CUDA cores (warp shuffles)  */
+    uint32_t upper_level_path;  /* 0 = levels above the products run on CUDA cores (warp shuffles);
+                                   1 = the scan over the 128 row totals is a tensor-core product on 8-bit limbs */
     uint64_t tiles;             /* 128 x 128-element tiles processed                                  */
     uint64_t mma_instructions;  /* tcgen05.mma instructions issued                                    */
     uint64_t sxs_products;      /* s x s-equivalent U_s products they amount to ( = padded n / s^2 )  */
@@ -180,6 +181,15 @@ tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned lim
 size_t tcu_sort_tmp_bytes(size_t n);
 tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_t n, void *d_tmp, size_t tmp_bytes,
                           void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Experiment knob (paper Section 2: "all numerical operations are multiplications between two
+ * square matrices"): path = 1 makes the following int8 scans of this process compute the scan over
+ * the 128 row totals of a tile - an upper level of the up-sweep, whose int32 operands are not a
+ * tensor-core input type - as a tcgen05 kind::i8 product of a strictly lower triangular all-ones
+ * matrix with the totals split into two signed 8-bit limbs, recombined exactly.  path = 0 (default)
+ * uses warp shuffles.  Results are identical; tcu_scan_stats_t.upper_level_path records the choice.
+ * Floating-point inputs always use path 0. */
+tcu_status_t tcu_scan_set_upper_level_path(int path);
 
 /* Experiment knob: run the following scans of this process on at most `max_ctas` persistent CTAs,
  * i.e. on that many SMs (0 restores the default, one CTA per SM).  One CTA owns one SM's tensor

@@ -56,6 +56,8 @@ _lib.tcu_sort_tmp_bytes.argtypes = [_sz]
 _lib.tcu_sort_tmp_bytes.restype = _sz
 _lib.tcu_sort_u32.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _sz, _vp]
 _lib.tcu_sort_u32.restype = _int
+_lib.tcu_scan_set_upper_level_path.argtypes = [_int]
+_lib.tcu_scan_set_upper_level_path.restype = _int
 _lib.tcu_scan_set_max_ctas.argtypes = [_int]
 _lib.tcu_scan_set_max_ctas.restype = _int
 _lib.tcu_scan_last_stats.argtypes = [ctypes.POINTER(TcuScanStats)]
@@ -132,6 +134,10 @@ def tcu_sort_tmp_bytes(n: int) -> int:
 
 def tcu_sort_u32(d_keys_in, d_keys_out, n: int, d_tmp, tmp_bytes: int, d_ws, ws_bytes: int, stream=0) -> int:
     return _lib.tcu_sort_u32(_p(d_keys_in), _p(d_keys_out), n, _p(d_tmp), tmp_bytes, _p(d_ws), ws_bytes, stream)
+
+
+def tcu_scan_set_upper_level_path(path: int) -> int:
+    return _lib.tcu_scan_set_upper_level_path(int(path))
 
 
 def tcu_scan_set_max_ctas(max_ctas: int) -> int:

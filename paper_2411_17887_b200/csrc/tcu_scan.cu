@@ -33,6 +33,7 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+std::atomic<int> g_upper_path{0};  // 0 = row totals scanned with warp shuffles, 1 = with a product on 8-bit limbs (int8 input only)
 std::atomic<int> g_max_ctas{0};   // 0 = one CTA per SM; otherwise the persistent grid is capped (scaling experiments)
 std::mutex g_stats_mutex;
 tcu_scan_stats_t g_stats;
@@ -148,7 +149,8 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     const int b_atoms = (seff * eb + 127) / 128;
     const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
     const uint32_t stage_bytes = kTileElems * eb;
-    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + 1024;  // + alignment slack
+    const bool upper_tc = (dt == TCU_I8_I32) && g_upper_path.load() == 1;
+    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? kUpperBytes : 0) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kUseInStages) in_stages = kUseInStages;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
@@ -162,9 +164,9 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     st.dtype = dt;
     st.exclusive = exclusive;
     st.variant = two_sweep ? 1 : 0;
-    st.upper_level_path = 0;
+    st.upper_level_path = upper_tc ? 1 : 0;
     st.tiles = tiles;
-    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32);  // U_s products + row-total products
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? 4 : 0));  // U_s products + row-total products
     st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
     // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
     // scan over the tiles (absent for a single tile), carry add
@@ -218,6 +220,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         prm.dtype = uint32_t(dt);
         prm.level0_only = level0 ? 1u : 0u;
         prm.prefilled = two_sweep ? 1u : 0u;
+        prm.upper_tc = upper_tc ? 1u : 0u;
         if (two_sweep) {
             // sweep 1: one total per tile; then their scan, written as the records sweep 2 looks back over
             const uint64_t valid = uint64_t(rows128) * kTileCols;
@@ -463,6 +466,12 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
         src = dst;
     }
+    return TCU_OK;
+}
+
+tcu_status_t tcu_scan_set_upper_level_path(int path) {
+    if (path != 0 && path != 1) return TCU_ERR_INVALID_ARG;
+    g_upper_path.store(path);
     return TCU_OK;
 }
 

@@ -82,6 +82,7 @@ constexpr uint32_t kPrefetchDist = TCU_PREFETCH_DIST;
 constexpr int kLookBack = TCU_LOOKBACK;
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
+constexpr int kUpperBytes = kAtomBytes + 16 * 128;   // limb variant: strictly lower triangular ones (128 x 128 int8) + limb operand
 constexpr int kEpilogueThreads = 128;
 // Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
 // 96 x 640 = 61440 registers), so 128 x (64 + 64 + 40 + kStoreGroups x kStoreRegs) must not exceed it:
@@ -151,6 +152,7 @@ struct alignas(64) ScanParams {
     uint32_t dtype;           // tcu_dtype_t
     uint32_t level0_only;     // debug: stop after the U_s product (no carries)
     uint32_t prefilled;       // two-sweep variant: the records already hold every tile's inclusive sum
+    uint32_t upper_tc;        // int8 only: scan the 128 row totals with a second triangular product on 8-bit limbs
 };
 
 // shared-memory bookkeeping (lives at the 1024-aligned base of dynamic shared memory)
@@ -172,6 +174,7 @@ struct SmemCtl {
     uint32_t epoch;
     uint32_t carry_in_bits;          // value at *carry_in (0 when there is none)
     uint64_t epoch_ready;            // thread 0 -> totals and look-back warps: epoch and carry_in_bits are written
+    uint64_t up_done;                // limb product of the row totals -> totals warps
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 2048;
@@ -423,6 +426,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *const_region = ones_region + kOnesBytes;
     uint8_t *in_ring = const_region + p.b_bytes;
     uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
+    uint8_t *upper_a = out_ring + kOutRingBytes;          // only present when p.upper_tc
+    uint8_t *upper_b = upper_a + kAtomBytes;
 
     WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
     uint8_t *records = reinterpret_cast<uint8_t *>(p.ws) + kHeaderBytes;
@@ -442,6 +447,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         prev_epoch = ld_relaxed_u32(&hdr->epoch);
 #endif
         mbar_init(smem_u32(&ctl->epoch_ready), 1);
+        mbar_init(smem_u32(&ctl->up_done), 1);
     }
     {
         // the barriers are the first kNumBarriers 64-bit words of the control block: one thread each
@@ -487,6 +493,14 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     *reinterpret_cast<uint16_t *>(const_region + off) = (p.dtype == 2) ? 0x3F80 : 0x3C00;
                 }
             }
+        }
+        if (IS_INT && p.upper_tc) {
+            // A[m][k] = 1 for k < m: its product with a column of row totals is their exclusive scan over the rows
+            for (int e = threadIdx.x; e < kTileRows * kTileRows; e += kThreads) {
+                const int m = e >> 7, k = e & 127;
+                upper_a[m * 128 + ((((k >> 4) ^ (m & 7))) << 4) + (k & 15)] = (k < m) ? 1 : 0;
+            }
+            for (int e = threadIdx.x; e < 16 * 128 / 4; e += kThreads) reinterpret_cast<uint32_t *>(upper_b)[e] = 0;
         }
         fence_proxy_async_smem();
     }
@@ -795,6 +809,48 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             tc_fence_after();
             const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
             tmem_ld_wait();
+            if (IS_INT && p.upper_tc) {
+                // Paper-faithful variant of this level: the scan over the 128 row totals is itself a product
+                // with a triangular all-ones matrix.  Row totals are int32, not a tensor-core input type, so
+                // each is split into two signed 8-bit limbs (total = 128 h + l, |total| <= 2^14), the limbs
+                // are scanned by one kind::i8 product, and the two results are recombined exactly.
+                const int32_t tot = int32_t(rowtot);
+                const uint32_t ub = smem_u32(upper_b);
+                const uint32_t off = ((r >> 4) << 4) + (r & 15);         // k = r inside a 128-byte row, before the swizzle
+                asm volatile("st.shared.u8 [%0], %1;" ::"r"(ub + 0 * 128 + ((((r >> 4) ^ 0) << 4) | (r & 15))), "r"(tot & 127) : "memory");
+                asm volatile("st.shared.u8 [%0], %1;" ::"r"(ub + 1 * 128 + ((((r >> 4) ^ 1) << 4) | (r & 15))), "r"((tot >> 7) & 0xFF) : "memory");
+                (void)off;
+                fence_proxy_async_smem();
+                named_barrier_sync(2, kEpilogueThreads);
+                if (r == 0) {
+                    tc_fence_after();
+                    const uint32_t idesc = make_idesc(0, kTotCols);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_issue<true>(tmem_base + kTotBase + tt * kTotCols, make_smem_desc(smem_u32(upper_a) + kk * 32),
+                                        make_smem_desc(ub + kk * 32), idesc, kk > 0 ? 1u : 0u);
+                    mma_commit(smem_u32(&ctl->up_done));
+                }
+                (void)w.wait(smem_u32(&ctl->up_done), j & 1);              // (a wait that ran out is caught by the next vote)
+                tc_fence_after();
+                const uint32_t d0 = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
+                const uint32_t d1 = tmem_ld1(lane_base + kTotBase + tt * kTotCols + 1);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(smem_u32(&ctl->tot_empty[tt]));            // the small accumulator may be refilled
+                const uint32_t exc_all = d0 + (d1 << 7);                   // sum of the totals of rows 0 .. r-1
+                rowpref[ts * kTileRows + r] = exc_all;
+                if (r == kTileRows - 1) {
+                    const CarryT a = CarryT(exc_all + rowtot);
+                    const bool first = (t % p.tiles_per_row == 0);
+                    const uint32_t status = first ? kStatusInclusive : kStatusPartial;
+                    if (!p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
+                    ctl->agg_slot[ts] = CO::enc(a);
+                }
+                mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
+                PROF_ADD(1);
+                continue;
+            }
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->tot_empty[tt]));                // the small accumulator may be refilled
             uint32_t inc = rowtot;                                    // inclusive scan across the warp's 32 rows

@@ -173,3 +173,24 @@ def test_result_does_not_depend_on_the_number_of_ctas(runner):
     finally:
         B.check(B.tcu_scan_set_max_ctas(0))
     assert B.tcu_scan_set_max_ctas(-1) == B.TCU_ERR_INVALID_ARG
+
+
+def test_row_total_scan_on_tensor_cores_gives_the_same_integers(runner):
+    # upper level as a triangular product on 8-bit limbs instead of warp shuffles (int8 input)
+    from paper_2411_17887_b200 import binding as B
+    from tests.gpu_util import check
+    try:
+        B.check(B.tcu_scan_set_upper_level_path(1))
+        for n, s in [(TILE, 16), (9 * TILE + 128 * 3 + 5, 64), (700 * TILE + 77, 16), (300 * TILE, 128)]:
+            x = gen("i8", n, 7000 + n % 313)
+            check(runner, x, "i8", s)
+            check(runner, x, "i8", s, True)
+            assert B.tcu_scan_last_stats()["upper_level_path"] == 1
+        extreme = np.full(5 * TILE, -128, np.int8)          # row totals of -2^14: the limb split at its limit
+        check(runner, extreme, "i8", 16)
+        check(runner, np.full(5 * TILE, 127, np.int8), "i8", 16)
+        check(runner, gen("f16", 3 * TILE, 5), "f16", 16)   # floating-point input keeps the shuffle path
+        assert B.tcu_scan_last_stats()["upper_level_path"] == 0
+    finally:
+        B.check(B.tcu_scan_set_upper_level_path(0))
+    assert B.tcu_scan_set_upper_level_path(2) == B.TCU_ERR_INVALID_ARG
