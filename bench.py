@@ -194,6 +194,18 @@ def run_ours(args):
     def step():
         B.check(B.tcu_scan_inclusive(d_in, d_out, n, B.TCU_I8_I32, S_TILE, ws_ptr, ws_bytes, stream))
 
+    if args.profile:
+        # the loop that is wrapped in ncu: optionally another input type, tile size or variant of the upper levels
+        B.check(B.tcu_scan_set_upper_level_path(args.upper_level_path))
+        B.check(B.tcu_scan_set_down_sweep_path(args.down_sweep_path))
+        if args.profile_dtype == "f16":
+            d_in = torch.from_numpy(inputs.f16_uniform((n,), -1.0, 1.0, cfg.index)).cuda()
+            d_out = torch.empty(n, dtype=torch.float32, device="cuda")
+        prof_dt = B.DTYPES[args.profile_dtype]
+
+        def step():  # noqa: F811
+            B.check(B.tcu_scan_inclusive(d_in, d_out, n, prof_dt, args.profile_s, ws_ptr, ws_bytes, stream))
+
     # ---- device-resident timing
     for _ in range(max(args.warmup, 3)):
         step()
@@ -211,8 +223,10 @@ def run_ours(args):
     if args.profile:
         if rank == 0:
             ms_step = ms_total / args.steps
-            print(json.dumps({"profile_run": True, "n": n, "ms_per_step": ms_step,
-                              "hbm_gb_per_s": BYTES_PER_ELEM * n / (ms_step * 1e-3) / 1e9}))
+            bpe = 5 if args.profile_dtype == "i8" else 6
+            print(json.dumps({"profile_run": True, "n": n, "dtype": args.profile_dtype, "s": args.profile_s,
+                              "upper_level_path": args.upper_level_path, "down_sweep_path": args.down_sweep_path,
+                              "ms_per_step": ms_step, "hbm_gb_per_s": bpe * n / (ms_step * 1e-3) / 1e9}))
         if sampler:
             sampler.stop()
         if world > 1:
@@ -295,6 +309,12 @@ def run_ours(args):
                 extras.append(time_extra(B, torch, "C3 with the scan over row totals as a tcgen05 product on 8-bit limbs (upper_level_path = 1)",
                                          d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes))
                 B.check(B.tcu_scan_set_upper_level_path(0))
+                # fp16, s = 128: carries added by a tensor-core product (the paper's B_s step) instead of vector adds
+                for path in (0, 1):
+                    B.check(B.tcu_scan_set_down_sweep_path(path))
+                    extras.append(time_extra(B, torch, f"fp16 n=2^28, s=128, down_sweep_path = {path}", xf, 1, 1 << 28, 1, 128,
+                                             False, ws_ptr, ws_bytes))
+                B.check(B.tcu_scan_set_down_sweep_path(0))
                 # application: radix sort of 2^24 keys by 32 one-bit splits, each an exclusive scan of int8 flags
                 ns = 1 << 24
                 keys = torch.randint(0, 1 << 31, (ns,), device="cuda", dtype=torch.int32, generator=g)
@@ -350,6 +370,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true", help="skip the timings of the other configurations")
+    ap.add_argument("--profile-dtype", default="i8", choices=["i8", "f16"], help="input type of the --profile loop")
+    ap.add_argument("--profile-s", type=int, default=16, help="tile size s of the --profile loop")
+    ap.add_argument("--upper-level-path", type=int, default=0, choices=[0, 1],
+                    help="1: scan the row totals with a tensor-core product on 8-bit limbs (int8 input)")
+    ap.add_argument("--down-sweep-path", type=int, default=0, choices=[0, 1],
+                    help="1: add the row carries with a tensor-core product (fp16 input, s = 128)")
     ap.add_argument("--sweep-ctas", action="store_true",
                     help="also time the headline scan on p = 1, 2, 4, ... persistent CTAs (one per SM) and report time vs p")
     ap.add_argument("--n-log2", type=int, default=28, help="log2 of the array length (28 = the headline workload)")

@@ -73,6 +73,7 @@ typedef struct {
                                    carry add), to be compared with the paper's 2 floor(log_s n)        */
     uint32_t depth_bound;       /* 2 floor(log_s cols), Corollary 1                                   */
     uint32_t grid, smem_bytes, in_stages, tail_elements;
+    uint32_t down_sweep_path;   /* 0 = carries added on the vector ALUs; 1 = by a tensor-core product        */
 } tcu_scan_stats_t;
 
 /* Bytes of device workspace needed to scan `rows` independent rows of `cols` elements
@@ -190,6 +191,14 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
  * uses warp shuffles.  Results are identical; tcu_scan_stats_t.upper_level_path records the choice.
  * Floating-point inputs always use path 0. */
 tcu_status_t tcu_scan_set_upper_level_path(int path);
+
+/* Experiment knob (paper Section 2, matrix B_s, and the discussion's remark that the tensor unit is
+ * used at O(1/s) in the down-sweep): path = 1 makes the following fp16 / bf16 scans with s = 128
+ * add each row's carry to the whole row by a tcgen05 product - accumulator += C * ones, C holding
+ * the carry split exactly into three bf16 terms - instead of one vector add per element.  Other
+ * dtypes and tile sizes ignore it.  Results satisfy the same tolerance;
+ * tcu_scan_stats_t.down_sweep_path records the choice. */
+tcu_status_t tcu_scan_set_down_sweep_path(int path);
 
 /* Experiment knob: run the following scans of this process on at most `max_ctas` persistent CTAs,
  * i.e. on that many SMs (0 restores the default, one CTA per SM).  One CTA owns one SM's tensor

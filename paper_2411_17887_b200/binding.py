@@ -31,7 +31,7 @@ class TcuScanStats(ctypes.Structure):
                 ("tiles", ctypes.c_uint64), ("mma_instructions", ctypes.c_uint64), ("sxs_products", ctypes.c_uint64),
                 ("levels_used", ctypes.c_uint32), ("depth_bound", ctypes.c_uint32),
                 ("grid", ctypes.c_uint32), ("smem_bytes", ctypes.c_uint32), ("in_stages", ctypes.c_uint32),
-                ("tail_elements", ctypes.c_uint32)]
+                ("tail_elements", ctypes.c_uint32), ("down_sweep_path", ctypes.c_uint32)]
 
 
 _vp, _sz, _int = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
@@ -56,6 +56,8 @@ _lib.tcu_sort_tmp_bytes.argtypes = [_sz]
 _lib.tcu_sort_tmp_bytes.restype = _sz
 _lib.tcu_sort_u32.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _sz, _vp]
 _lib.tcu_sort_u32.restype = _int
+_lib.tcu_scan_set_down_sweep_path.argtypes = [_int]
+_lib.tcu_scan_set_down_sweep_path.restype = _int
 _lib.tcu_scan_set_upper_level_path.argtypes = [_int]
 _lib.tcu_scan_set_upper_level_path.restype = _int
 _lib.tcu_scan_set_max_ctas.argtypes = [_int]
@@ -134,6 +136,10 @@ def tcu_sort_tmp_bytes(n: int) -> int:
 
 def tcu_sort_u32(d_keys_in, d_keys_out, n: int, d_tmp, tmp_bytes: int, d_ws, ws_bytes: int, stream=0) -> int:
     return _lib.tcu_sort_u32(_p(d_keys_in), _p(d_keys_out), n, _p(d_tmp), tmp_bytes, _p(d_ws), ws_bytes, stream)
+
+
+def tcu_scan_set_down_sweep_path(path: int) -> int:
+    return _lib.tcu_scan_set_down_sweep_path(int(path))
 
 
 def tcu_scan_set_upper_level_path(path: int) -> int:

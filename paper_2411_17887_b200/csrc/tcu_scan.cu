@@ -34,6 +34,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 std::atomic<int> g_upper_path{0};  // 0 = row totals scanned with warp shuffles, 1 = with a product on 8-bit limbs (int8 input only)
+std::atomic<int> g_down_path{0};   // 0 = carries added on the vector ALUs, 1 = by a tensor-core product (16-bit input, s = 128 only)
 std::atomic<int> g_max_ctas{0};   // 0 = one CTA per SM; otherwise the persistent grid is capped (scaling experiments)
 std::mutex g_stats_mutex;
 tcu_scan_stats_t g_stats;
@@ -150,7 +151,9 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
     const uint32_t stage_bytes = kTileElems * eb;
     const bool upper_tc = (dt == TCU_I8_I32) && g_upper_path.load() == 1;
-    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? kUpperBytes : 0) + 1024;  // + alignment slack
+    const bool down_tc = (dt != TCU_I8_I32) && s == 128 && !level0 && g_down_path.load() == 1;
+    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? kUpperBytes : 0) +
+                         (down_tc ? kDownBytes : 0) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kUseInStages) in_stages = kUseInStages;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
@@ -165,8 +168,9 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     st.exclusive = exclusive;
     st.variant = two_sweep ? 1 : 0;
     st.upper_level_path = upper_tc ? 1 : 0;
+    st.down_sweep_path = down_tc ? 1 : 0;
     st.tiles = tiles;
-    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? 4 : 0));  // U_s products + row-total products
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? 4 : 0) + (down_tc ? 1 : 0));  // U_s products + row-total products
     st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
     // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
     // scan over the tiles (absent for a single tile), carry add
@@ -221,6 +225,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         prm.level0_only = level0 ? 1u : 0u;
         prm.prefilled = two_sweep ? 1u : 0u;
         prm.upper_tc = upper_tc ? 1u : 0u;
+        prm.down_tc = down_tc ? 1u : 0u;
         if (two_sweep) {
             // sweep 1: one total per tile; then their scan, written as the records sweep 2 looks back over
             const uint64_t valid = uint64_t(rows128) * kTileCols;
@@ -466,6 +471,12 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
         src = dst;
     }
+    return TCU_OK;
+}
+
+tcu_status_t tcu_scan_set_down_sweep_path(int path) {
+    if (path != 0 && path != 1) return TCU_ERR_INVALID_ARG;
+    g_down_path.store(path);
     return TCU_OK;
 }
 

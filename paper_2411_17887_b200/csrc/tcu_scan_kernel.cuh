@@ -82,6 +82,7 @@ constexpr uint32_t kPrefetchDist = TCU_PREFETCH_DIST;
 constexpr int kLookBack = TCU_LOOKBACK;
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
+constexpr int kDownBytes = (kStoreGroups + 1) * kAtomBytes;   // carry-product variant: one carry operand per store group + a ones operand
 constexpr int kUpperBytes = kAtomBytes + 16 * 128;   // limb variant: strictly lower triangular ones (128 x 128 int8) + limb operand
 constexpr int kEpilogueThreads = 128;
 // Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
@@ -152,6 +153,7 @@ struct alignas(64) ScanParams {
     uint32_t dtype;           // tcu_dtype_t
     uint32_t level0_only;     // debug: stop after the U_s product (no carries)
     uint32_t prefilled;       // two-sweep variant: the records already hold every tile's inclusive sum
+    uint32_t down_tc;         // 16-bit input, s = 128 only: add the row carries with a tensor-core product (B_s-style down-sweep)
     uint32_t upper_tc;        // int8 only: scan the 128 row totals with a second triangular product on 8-bit limbs
 };
 
@@ -175,6 +177,7 @@ struct SmemCtl {
     uint32_t carry_in_bits;          // value at *carry_in (0 when there is none)
     uint64_t epoch_ready;            // thread 0 -> totals and look-back warps: epoch and carry_in_bits are written
     uint64_t up_done;                // limb product of the row totals -> totals warps
+    uint64_t down_done[kStoreGroups];   // carry product -> store warps of a group
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 2048;
@@ -428,6 +431,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
     uint8_t *upper_a = out_ring + kOutRingBytes;          // only present when p.upper_tc
     uint8_t *upper_b = upper_a + kAtomBytes;
+    uint8_t *down_a = out_ring + kOutRingBytes;           // only present when p.down_tc (never together with upper_tc)
+    uint8_t *down_b = down_a + kStoreGroups * kAtomBytes;
 
     WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
     uint8_t *records = reinterpret_cast<uint8_t *>(p.ws) + kHeaderBytes;
@@ -448,6 +453,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 #endif
         mbar_init(smem_u32(&ctl->epoch_ready), 1);
         mbar_init(smem_u32(&ctl->up_done), 1);
+        for (int g = 0; g < kStoreGroups; ++g) mbar_init(smem_u32(&ctl->down_done[g]), 1);
     }
     {
         // the barriers are the first kNumBarriers 64-bit words of the control block: one thread each
@@ -493,6 +499,12 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     *reinterpret_cast<uint16_t *>(const_region + off) = (p.dtype == 2) ? 0x3F80 : 0x3C00;
                 }
             }
+        }
+        if (!IS_INT && p.down_tc) {
+            // carry operands start as zeros (only 3 of the 16 K-entries of a row are ever written); the other
+            // operand is all ones in bf16
+            for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 4; e += kThreads) reinterpret_cast<uint32_t *>(down_a)[e] = 0;
+            for (int e = threadIdx.x; e < kAtomBytes / 4; e += kThreads) reinterpret_cast<uint32_t *>(down_b)[e] = 0x3F803F80u;
         }
         if (IS_INT && p.upper_tc) {
             // A[m][k] = 1 for k < m: its product with a column of row totals is their exclusive scan over the rows
@@ -929,6 +941,32 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (level0) base = 0;
             uint32_t run = base;                                      // sum of everything before the current chunk
             uint32_t prev = base;                                     // value of the element to the left (exclusive form)
+            if (!IS_INT && S == 128 && p.down_tc && !level0) {
+                // Paper-faithful variant of the down-sweep (the B_s product: one carry added to a whole vector):
+                // the accumulator gets D += C * 1, where row r of C holds the row's carry split exactly into
+                // three bf16 terms and 1 is an all-ones operand.  128 x 128 x 16 multiply-adds for 16 Ki useful
+                // additions - the low utilisation the paper's discussion predicts for this step.
+                const float b0 = __uint_as_float(base);
+                const uint32_t hi = __float_as_uint(b0) & 0xFFFF0000u;
+                const float r1 = b0 - __uint_as_float(hi);
+                const uint32_t mid = __float_as_uint(r1) & 0xFFFF0000u;
+                const float r2 = r1 - __uint_as_float(mid);
+                const uint32_t lo = __float_as_uint(r2) & 0xFFFF0000u;             // r2 has at most 8 significant bits
+                const uint32_t da = smem_u32(down_a) + group * kAtomBytes;
+                const uint32_t row_addr = da + r * 128 + ((0 ^ (r & 7)) << 4);       // K entries 0..7 of row r
+                asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(row_addr), "r"((hi >> 16) | mid), "r"(lo >> 16) : "memory");
+                fence_proxy_async_smem();
+                named_barrier_sync(3 + group, kEpilogueThreads);
+                if (wq == 0 && lane == 0) {
+                    tc_fence_after();
+                    mma_issue<false>(tmem_base + slot * kTileCols, make_smem_desc(da), make_smem_desc(smem_u32(down_b)),
+                                     make_idesc(2, kTileCols), 1u);
+                    mma_commit(smem_u32(&ctl->down_done[group]));
+                }
+                if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->down_done[group]), (j / kStoreGroups) & 1))) break;
+                tc_fence_after();
+                run = 0;                                              // the carry is inside the accumulator now
+            }
             const uint32_t row0 = lt * kTileRows + wq * 32;           // first 128-element row of this warp's part of the tile
             uint32_t *const gbase = out32 + size_t(scan_row) * p.scan_pitch + size_t(row0) * kTileCols + piece * 4;
             const int rows_here = int(p.rows128) - int(row0);         // rows of this part that exist (ragged last tile)

@@ -194,3 +194,24 @@ def test_row_total_scan_on_tensor_cores_gives_the_same_integers(runner):
     finally:
         B.check(B.tcu_scan_set_upper_level_path(0))
     assert B.tcu_scan_set_upper_level_path(2) == B.TCU_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_down_sweep_as_a_tensor_core_product(runner, dtype):
+    # the carry of every row added by accumulator += C * ones (C = carry in three bf16 terms) instead of vector adds
+    from paper_2411_17887_b200 import binding as B
+    from tests.gpu_util import check
+    try:
+        B.check(B.tcu_scan_set_down_sweep_path(1))
+        for n in (TILE, 9 * TILE + 128 * 3 + 5, 400 * TILE + 77):
+            for exclusive in (False, True):
+                check(runner, gen(dtype, n, 8000 + n % 211), dtype, 128, exclusive)
+                assert B.tcu_scan_last_stats()["down_sweep_path"] == 1
+        got = runner.run(np.ones(1 << 22, np.float16), "f16", 128)          # integers up to 2^22: must stay exact
+        assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
+        check(runner, gen(dtype, 5 * TILE, 3), dtype, 16)                   # other tile sizes ignore the knob
+        assert B.tcu_scan_last_stats()["down_sweep_path"] == 0
+        check(runner, gen("i8", 5 * TILE, 4), "i8", 128)
+        assert B.tcu_scan_last_stats()["down_sweep_path"] == 0
+    finally:
+        B.check(B.tcu_scan_set_down_sweep_path(0))
