@@ -7,7 +7,7 @@ arrays.  It shares no code with the CUDA library.
 Definition followed (paper, Section 1, notation paragraph): "prefix sum" is the
 inclusive prefix sum under +; the exclusive form shifts the result right by one
 and puts the identity 0 in front.  Input types and the widening rules are not
-in the paper; they are this build's: int8 is summed exactly in int64 and then
+in the paper; they are this library's: int8 is summed exactly in int64 and then
 reported modulo 2**32 as a two's-complement int32, fp16 / bf16 are widened
 exactly to fp64 and summed in fp64.
 """
