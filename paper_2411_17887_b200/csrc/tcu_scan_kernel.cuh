@@ -34,6 +34,12 @@ namespace tcu {
 #ifndef TCU_PREFETCH_DIST
 #define TCU_PREFETCH_DIST 256   // tiles ahead of the claimed one that are prefetched into L2 (0 = off)
 #endif
+#ifndef TCU_ST_HINT
+#define TCU_ST_HINT 0           // output stores: 0 = plain, 1 = st.global.cs (streaming), 2 = st.global.L1::no_allocate
+#endif
+#ifndef TCU_LD_HINT
+#define TCU_LD_HINT 0           // input TMA loads: 1 = L2 evict-first hint (every tile is read once)
+#endif
 #ifndef TCU_PDL
 #define TCU_PDL 1               // programmatic dependent launch: set-up overlaps the tail of the previous kernel in the stream
 #endif
@@ -217,6 +223,15 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+#if TCU_LD_HINT
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
+        : "memory");
+    return;
+#endif
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
@@ -322,7 +337,13 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t &a, uint32_
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void st_global_v4(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+#if TCU_ST_HINT == 1
+    asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+#elif TCU_ST_HINT == 2
+    asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+#else
     asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+#endif
 }
 __device__ __forceinline__ void ld_record(const void *p, uint64_t &flag, uint64_t &val) {
     asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(flag), "=l"(val) : "l"(p) : "memory");
