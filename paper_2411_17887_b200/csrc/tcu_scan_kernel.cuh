@@ -53,7 +53,7 @@ namespace tcu {
 #define TCU_SETMAXNREG 1        // move registers from the control warps to the store warps
 #endif
 #ifndef TCU_LOOKBACK
-#define TCU_LOOKBACK 2          // windows of 32 records fetched per look-back round
+#define TCU_LOOKBACK 1          // windows of 32 records fetched per look-back round
 #endif
 #ifndef TCU_STATIC_TILES
 #define TCU_STATIC_TILES 0      // 1 = tile j of CTA b is b + j * gridDim.x instead of the next ticket
@@ -464,8 +464,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 
     // ---- set-up
     PROF_STAMP(0);
-    uint32_t first_ticket = 0;                 // (thread 0 only) claimed before anything else, so that the round trip
-    uint32_t prev_epoch = 0;                   // of the atomic and of the epoch read overlap the rest of the set-up
+    uint32_t first_ticket = 0;                 // (thread 0 only) first tile of this CTA
+    uint32_t prev_epoch = 0;                   // (thread 0 only) launches completed on the workspace so far
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&p.tmap_in)) : "memory");
 #if !TCU_PDL
