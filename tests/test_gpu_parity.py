@@ -215,3 +215,29 @@ def test_down_sweep_as_a_tensor_core_product(runner, dtype):
         assert B.tcu_scan_last_stats()["down_sweep_path"] == 0
     finally:
         B.check(B.tcu_scan_set_down_sweep_path(0))
+
+
+def test_many_back_to_back_launches_agree(runner):
+    # consecutive launches overlap their set-up with the previous kernel's tail and reuse one workspace:
+    # every one of them must reproduce the integers of the first, whatever the number of CTAs
+    from paper_2411_17887_b200 import binding as B
+    from oracle import scan_oracle as so
+    from tests.gpu_util import to_device
+    n = 600 * TILE + 77
+    x = gen("i8", n, 123)
+    ref = torch.from_numpy(so.scan(x, "i8")["y32"]).cuda()
+    d_in = to_device(x, "i8")
+    outs = [torch.empty(n, dtype=torch.int32, device="cuda") for _ in range(4)]
+    try:
+        for it in range(120):
+            if it % 30 == 0:
+                B.check(B.tcu_scan_set_max_ctas([0, 5, 77, 148][it // 30]))
+            out = outs[it % 4]
+            B.check(B.tcu_scan_inclusive(d_in, out, n, B.TCU_I8_I32, 16, runner.ws_ptr, runner.ws_bytes, 0))
+            if it % 4 == 3:
+                for o in outs:
+                    assert torch.equal(o, ref)
+                    o.fill_(-1)
+    finally:
+        B.check(B.tcu_scan_set_max_ctas(0))
+    B.check(B.tcu_scan_device_status(runner.ws_ptr, 0))
