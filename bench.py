@@ -155,7 +155,10 @@ def time_extra(B, torch, name, x, rows, cols, dt, s, exclusive, ws_ptr, ws_bytes
     ms = e0.elapsed_time(e1) / reps
     nbytes = rows * cols * ((1 if dt == 0 else 2) + 4)
     del out
-    return {"workload": name, "ms": ms, "elements_per_s": rows * cols / (ms * 1e-3), "GB_per_s": nbytes / (ms * 1e-3) / 1e9}
+    st = B.tcu_scan_last_stats()
+    return {"workload": name, "ms": ms, "elements_per_s": rows * cols / (ms * 1e-3), "GB_per_s": nbytes / (ms * 1e-3) / 1e9,
+            "levels_used": st["levels_used"], "depth_bound_2floor_log_s_n": st["depth_bound"],
+            "sxs_products": st["sxs_products"], "n_over_s2": rows * cols // (s * s), "mma_instructions": st["mma_instructions"]}
 
 
 def run_ours(args):
