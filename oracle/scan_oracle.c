@@ -76,3 +76,20 @@ void oracle_scan_rows_f64(const double *x, size_t rows, size_t cols, int exclusi
     for (size_t r = 0; r < rows; ++r)
         oracle_scan_f64(x + r * cols, cols, exclusive, 0.0, y + r * cols, a ? a + r * cols : (double *)0);
 }
+
+/* Segmented form: the array is cut at offsets[0] = 0 <= offsets[1] <= ... <= offsets[num_segments] = n and
+ * every piece [offsets[k], offsets[k+1]) is scanned on its own, from zero (paper, Section 2.2 steps 1-4 build
+ * the scan of a long array out of independent scans of consecutive segments plus their totals; here the
+ * totals are not carried over, because the segments are separate problems).  Empty pieces are allowed. */
+void oracle_scan_segments_i8_i64(const int8_t *x, const uint64_t *offsets, size_t num_segments, int exclusive, int64_t *y)
+{
+    for (size_t k = 0; k < num_segments; ++k)
+        oracle_scan_i8_i64(x + offsets[k], (size_t)(offsets[k + 1] - offsets[k]), exclusive, 0, y + offsets[k]);
+}
+
+void oracle_scan_segments_f64(const double *x, const uint64_t *offsets, size_t num_segments, int exclusive, double *y, double *a)
+{
+    for (size_t k = 0; k < num_segments; ++k)
+        oracle_scan_f64(x + offsets[k], (size_t)(offsets[k + 1] - offsets[k]), exclusive, 0.0, y + offsets[k],
+                        a ? a + offsets[k] : (double *)0);
+}

@@ -36,6 +36,10 @@ def _load():
         lib.oracle_scan_rows_i8_i64.restype = None
         lib.oracle_scan_rows_f64.argtypes = [vp, c_sz, c_sz, c_int, vp, vp]
         lib.oracle_scan_rows_f64.restype = None
+        lib.oracle_scan_segments_i8_i64.argtypes = [vp, vp, c_sz, c_int, vp]
+        lib.oracle_scan_segments_i8_i64.restype = None
+        lib.oracle_scan_segments_f64.argtypes = [vp, vp, c_sz, c_int, vp, vp]
+        lib.oracle_scan_segments_f64.restype = None
         _lib = lib
     return _lib
 
@@ -125,6 +129,28 @@ def scan(x: np.ndarray, dtype: str, exclusive: bool = False):
         y = scan_i8(x, exclusive)
         return {"y": y, "y32": wrap_int32(y)}
     y, a = scan_f64(widen(x, dtype), exclusive)
+    return {"y": y, "a": a}
+
+
+def scan_segments(x: np.ndarray, dtype: str, offsets, exclusive: bool = False):
+    """Segmented scan of a 1-D input: piece k is x[offsets[k]:offsets[k+1]], scanned from zero on its own.
+
+    ``offsets`` has one more entry than there are pieces, starts at 0, ends at len(x) and never decreases.
+    Returns the same dict as ``scan``; "a" restarts with every piece as well.
+    """
+    off = np.ascontiguousarray(offsets, dtype=np.uint64)
+    assert x.ndim == 1 and off.ndim == 1 and off.size >= 1
+    assert int(off[0]) == 0 and int(off[-1]) == x.size and bool((off[1:] >= off[:-1]).all())
+    lib = _load()
+    if dtype == "i8":
+        xi = np.ascontiguousarray(x, dtype=np.int8)
+        y = np.empty(xi.shape, dtype=np.int64)
+        lib.oracle_scan_segments_i8_i64(_ptr(xi), _ptr(off), off.size - 1, int(exclusive), _ptr(y))
+        return {"y": y, "y32": wrap_int32(y)}
+    x64 = widen(x, dtype)
+    y = np.empty(x64.shape, dtype=np.float64)
+    a = np.empty(x64.shape, dtype=np.float64)
+    lib.oracle_scan_segments_f64(_ptr(x64), _ptr(off), off.size - 1, int(exclusive), _ptr(y), _ptr(a))
     return {"y": y, "a": a}
 
 

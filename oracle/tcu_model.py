@@ -29,16 +29,17 @@ Passages followed:
 Readings taken where the text leaves a choice (each is also listed in the
 design notes of the repository):
 
-* The constant matrix multiplies from the left (Section 2: "the matrix product
-  L_s w").
+* The constant matrix multiplies from the left (Section 2 describes the local
+  prefix sum as L_s applied to a column vector w).
 * Slice lengths are the true lengths ceil((n - start)/step); the floor
   expressions in the proof of Lemma 1 are one short for some t, which does not
   affect the lemma's bounds.
 * Products are counted with the tensor view, ceil(m/s^2) per round (Lemma 1);
   latency is counted with the stacked view, one invocation per round
   (Theorem 1).
-* Section 2.2 step 2 says "maximum values of each segment"; the value meant is
-  the last entry of the segment after its up-sweep, i.e. the segment total.
+* Section 2.2 step 2 asks for the largest value of each segment; the value meant
+  is the last entry of the segment after its up-sweep, i.e. the segment total
+  (a literal maximum would be wrong for signed input).
 * Section 2.2 step 3: q is the smallest integer with (actual number of
   segments) <= s^q, rather than the worst case k_1 (s-1) <= s^q.
 * Section 2.2 step 4: a segment of length m that receives a carry is viewed as
@@ -58,18 +59,17 @@ import numpy as np
 
 # --------------------------------------------------------------------------- constants
 def L_matrix(s: int, dtype=np.int64) -> np.ndarray:
-    """L_s: lower-triangular all-ones s x s matrix, diagonal included (Section 1)."""
-    return np.tril(np.ones((s, s), dtype=dtype))
+    """L_s: entry (i, j) is 1 when j <= i, else 0 (Section 1, notation): L_s w is the
+    inclusive prefix sum of a column vector w."""
+    i, j = np.indices((s, s))
+    return (j <= i).astype(dtype)
 
 
 def B_matrix(s: int, dtype=np.int64) -> np.ndarray:
-    """B_s: identity whose first column is all ones (displayed equation of Section 2).
-
-    B_s [alpha; q] = [alpha; q + alpha 1], the scalar/vector add.
-    """
-    b = np.eye(s, dtype=dtype)
-    b[:, 0] = 1
-    return b
+    """B_s: entry (i, j) is 1 on the diagonal and in column 0, else 0 (displayed equation
+    of Section 2): B_s [alpha; q] = [alpha; q + alpha 1], the scalar/vector add."""
+    i, j = np.indices((s, s))
+    return ((j == i) | (j == 0)).astype(dtype)
 
 
 # --------------------------------------------------------------------------- counters
@@ -91,7 +91,7 @@ class Counters:
 
 
 def _is_L(A: np.ndarray) -> bool:
-    return bool(np.array_equal(A, np.tril(np.ones_like(A))))
+    return bool(np.array_equal(A, L_matrix(A.shape[0], A.dtype)))
 
 
 # --------------------------------------------------------------------------- BatchMatMul
@@ -142,6 +142,26 @@ def exact_log(n: int, s: int) -> Optional[int]:
     return k if p == n else None
 
 
+@dataclass(frozen=True)
+class Round:
+    """One batched-product round of Algorithm 1: the sub-vector x[first::stride] is replaced by
+    BatchMatMul(sub-vector, operand), operand being "L" (up-sweep) or "B" (down-sweep)."""
+    first: int
+    stride: int
+    operand: str
+
+
+def algorithm1_rounds(k: int, s: int) -> List[Round]:
+    """The schedule of Algorithm 1 for n = s^k.  Up-sweep, level t = 0 .. k-1: the entries that end a
+    block of s^t elements (positions s^t - 1, 2 s^t - 1, ...) are scanned in groups of s.  Down-sweep,
+    level t = k-1 .. 1: starting at the end of the first block of s^t elements, the entries that end a
+    block of s^(t-1) elements are taken; every group of s begins with a finished prefix, which B_s adds
+    to the s - 1 block ends behind it."""
+    up = [Round(s ** t - 1, s ** t, "L") for t in range(k)]
+    down = [Round(s ** t - 1, s ** (t - 1), "B") for t in range(k - 1, 0, -1)]
+    return up + down
+
+
 def matmul_scan(x: np.ndarray, s: int, counters: Optional[Counters] = None,
                 trace: Optional[list] = None, up_sweep_only: bool = False,
                 count_rounds: bool = True) -> np.ndarray:
@@ -149,51 +169,45 @@ def matmul_scan(x: np.ndarray, s: int, counters: Optional[Counters] = None,
 
     ``trace`` (a list) receives a copy of x after every round.
     """
-    x = np.array(x, copy=True)
-    n = len(x)
-    k = exact_log(n, s)
+    state = np.array(x, copy=True)
+    k = exact_log(len(state), s)
     if k is None:
-        raise ValueError(f"Algorithm 1 needs len(x) = s^k, got n={n}, s={s}")
-    Ls, Bs = L_matrix(s, x.dtype), B_matrix(s, x.dtype)
-    for t in range(k):                                   # 1st phase (up-sweep)
-        start, step = s ** t - 1, s ** t
-        y = x[start::step]
-        z = batch_matmul(y, Ls, counters)
-        x[start::step] = z
+        raise ValueError(f"Algorithm 1 needs len(x) = s^k, got n={len(state)}, s={s}")
+    operands = {"L": L_matrix(s, state.dtype), "B": B_matrix(s, state.dtype)}
+    for rnd in algorithm1_rounds(k, s):
+        if up_sweep_only and rnd.operand == "B":
+            break
+        picked = slice(rnd.first, None, rnd.stride)
+        state[picked] = batch_matmul(state[picked], operands[rnd.operand], counters)
         if counters is not None and count_rounds:
             counters.rounds += 1
         if trace is not None:
-            trace.append(x.copy())
-    if up_sweep_only:
-        return x
-    for t in range(k - 1, 0, -1):                        # 2nd phase (down-sweep)
-        start, step = s ** t - 1, s ** (t - 1)
-        y = x[start::step]
-        z = batch_matmul(y, Bs, counters)
-        x[start::step] = z
-        if counters is not None and count_rounds:
-            counters.rounds += 1
-        if trace is not None:
-            trace.append(x.copy())
-    return x
+            trace.append(state.copy())
+    return state
 
 
 # --------------------------------------------------------------------------- Algorithm 2
 def matmul_scan_recursive(x: np.ndarray, s: int, counters: Optional[Counters] = None) -> np.ndarray:
-    """MatMulScanRecursive(x, s) of Algorithm 2.  Rounds are not counted here
-    (the recursion interleaves them); products and additions are."""
-    z = batch_matmul(np.array(x, copy=True), L_matrix(s, np.asarray(x).dtype), counters)
-    return _recurse(z, s, counters)
+    """MatMulScanRecursive(x, s) of Algorithm 2: local scans of all chunks first, then the recursive
+    procedure on the result.  Rounds are not counted here (the recursion interleaves them); products
+    and additions are."""
+    x = np.asarray(x)
+    local = batch_matmul(np.array(x, copy=True), L_matrix(s, x.dtype), counters)
+    return _finish_from_chunk_scans(local, s, counters)
 
 
-def _recurse(z: np.ndarray, s: int, counters: Optional[Counters]) -> np.ndarray:
-    if len(z) <= s:                                      # termination criterion
-        return z
-    start = s - 1
-    z[start::s] = batch_matmul(z[start::s], L_matrix(s, z.dtype), counters)
-    z[start::s] = _recurse(z[start::s].copy(), s, counters)
-    z[start:] = batch_matmul(z[start:], B_matrix(s, z.dtype), counters)
-    return z
+def _finish_from_chunk_scans(v: np.ndarray, s: int, counters: Optional[Counters]) -> np.ndarray:
+    """Algorithm 2's recursive procedure.  On entry every chunk of s entries of v holds its own scan,
+    so the chunk totals sit at positions s-1, 2s-1, ...  A vector of at most s entries is already done.
+    Otherwise: scan the chunk totals (their own chunk scans by one product, the rest by recursion),
+    write them back, and let B_s add each finished total to the s - 1 entries that follow it."""
+    if len(v) <= s:
+        return v
+    ends = slice(s - 1, None, s)
+    totals = batch_matmul(v[ends], L_matrix(s, v.dtype), counters)
+    v[ends] = _finish_from_chunk_scans(totals, s, counters)
+    v[s - 1:] = batch_matmul(v[s - 1:], B_matrix(s, v.dtype), counters)
+    return v
 
 
 # --------------------------------------------------------------------------- Section 2.2
@@ -311,16 +325,9 @@ def corollary1_depth_bound(n: int, s: int) -> int:
 
 # --------------------------------------------------------------------------- counts without data
 def _alg1_call_lengths(n: int, s: int) -> List[int]:
-    """Lengths m of the vectors handed to BatchMatMul by Algorithm 1, in order."""
-    k = exact_log(n, s)
-    lens = []
-    for t in range(k):
-        start, step = s ** t - 1, s ** t
-        lens.append(-(-(n - start) // step))
-    for t in range(k - 1, 0, -1):
-        start, step = s ** t - 1, s ** (t - 1)
-        lens.append(-(-(n - start) // step))
-    return lens
+    """Lengths m of the vectors handed to BatchMatMul by Algorithm 1, in order (the number of
+    positions first, first + stride, ... below n)."""
+    return [-(-(n - rnd.first) // rnd.stride) for rnd in algorithm1_rounds(exact_log(n, s), s)]
 
 
 def model_counts(n: int, s: int) -> GeneralReport:

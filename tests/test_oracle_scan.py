@@ -89,10 +89,70 @@ def test_rows_are_independent():
     for r in range(7):
         assert np.array_equal(y[r], np.cumsum(x[r].astype(np.int64)))
     xb = inputs.bf16_normal((5, 77), 11)
-    yb, ab = so.scan_f64(so.widen(xb, "bf16"))
     wide = so.bf16_bits_to_f64(xb)
+    yb, ab = so.scan_f64(so.widen(xb, "bf16"))
     for r in range(5):
         assert np.array_equal(yb[r], np.cumsum(wide[r]))
+        # the running sum of |x| that scales the tolerance restarts with every row as well
+        assert np.array_equal(ab[r], np.cumsum(np.abs(wide[r])))
+        assert ab[r][0] == abs(wide[r][0]) and (np.diff(ab[r]) >= 0).all()
+    yex, aex = so.scan_f64(so.widen(xb, "bf16"), exclusive=True)
+    for r in range(5):
+        assert yex[r].tolist() == [0.0] + np.cumsum(wide[r]).tolist()[:-1]
+        assert aex[r].tolist() == [0.0] + np.cumsum(np.abs(wide[r])).tolist()[:-1]
+
+
+def test_float_init_carries_over_pieces():
+    # scanning two halves, the second started from the first half's last value, reproduces the whole
+    # scan bit for bit (the additions happen in the same order); `a` never includes init
+    x = so.widen(inputs.f16_uniform(1000, -1.0, 1.0, 12), "f16")
+    whole, a_whole = so.scan_f64(x)
+    first, a_first = so.scan_f64(x[:400])
+    second, a_second = so.scan_f64(x[400:], init=float(first[-1]))
+    assert np.array_equal(np.concatenate([first, second]), whole)
+    assert np.array_equal(a_second, np.cumsum(np.abs(x[400:])))
+    assert np.allclose(np.concatenate([a_first, a_second + a_first[-1]]), a_whole, rtol=1e-14, atol=0)
+    # exclusive form: y[0] is init itself, and the chain continues from init + x[0]
+    ex, a_ex = so.scan_f64(x[400:], exclusive=True, init=float(first[-1]))
+    assert ex[0] == first[-1] and ex[1] == first[-1] + x[400] and a_ex[0] == 0.0
+    assert np.array_equal(ex[1:], second[:-1])
+    # a closed form: constant input 0.5 from init 10 is exactly 10 + (i + 1) / 2
+    y, a = so.scan_f64(np.full(64, 0.5), init=10.0)
+    assert y.tolist() == [10.0 + (i + 1) / 2 for i in range(64)] and a.tolist() == [(i + 1) / 2 for i in range(64)]
+
+
+def _segments_by_definition(x, offsets, exclusive):
+    """Every output computed on its own: the sum over the part of its segment before it (brute force)."""
+    out = [0] * len(x)
+    for k in range(len(offsets) - 1):
+        lo, hi = int(offsets[k]), int(offsets[k + 1])
+        for i in range(lo, hi):
+            acc = 0
+            for j in range(lo, i if exclusive else i + 1):
+                acc = acc + x[j]
+            out[i] = acc
+    return out
+
+
+@pytest.mark.parametrize("exclusive", [False, True])
+def test_segmented_scan_brute_force(exclusive):
+    # empty segments, segments of one element, a long one; integer and floating point
+    offsets = [0, 0, 1, 1, 4, 20, 20, 21, 64]
+    x = inputs.int8_uniform(64, -127, 127, 13)
+    r = so.scan_segments(x, "i8", offsets, exclusive)
+    assert r["y"].tolist() == _segments_by_definition([int(v) for v in x], offsets, exclusive)
+    xf = inputs.f16_uniform(64, -1.0, 1.0, 14)
+    rf = so.scan_segments(xf, "f16", offsets, exclusive)
+    vals = [float(v) for v in xf]
+    assert rf["y"].tolist() == _segments_by_definition(vals, offsets, exclusive)
+    assert rf["a"].tolist() == _segments_by_definition([abs(v) for v in vals], offsets, exclusive)
+    # one segment is the plain scan; one segment per element gives x itself (inclusive) or zeros (exclusive)
+    assert np.array_equal(so.scan_segments(x, "i8", [0, 64], exclusive)["y"], so.scan_i8(x, exclusive))
+    single = so.scan_segments(x, "i8", list(range(65)), exclusive)["y"]
+    assert np.array_equal(single, np.zeros(64, np.int64) if exclusive else x.astype(np.int64))
+    # dense rows are the special case of equal segments
+    rows = so.scan_segments(x, "i8", [0, 16, 32, 48, 64], exclusive)["y"]
+    assert np.array_equal(rows.reshape(4, 16), so.scan_i8(x.reshape(4, 16), exclusive))
 
 
 def test_int32_wrap():

@@ -88,6 +88,33 @@ def test_lemma1_depth_and_products(s, k):
     assert c.tcu_time(0) <= 4 * n + 2 * s * k
 
 
+@pytest.mark.parametrize("s,k", [(3, 1), (3, 4), (4, 3), (5, 3), (7, 2), (16, 2), (16, 3)])
+def test_exact_work_of_both_sweeps(s, k):
+    # Additions on real data, counted from the structure of Algorithm 1 (proof of Lemma 1) for n = s^k.
+    # Up-sweep round t scans n / s^(t+1) full groups of s entries, s(s-1)/2 additions each: in total
+    # (s-1)/2 * (n + n/s + ... + s) = s (n - 1) / 2.  Down-sweep round t works on the block ends of size
+    # s^(t-1) from position s^t - 1 on, s^(k-t+1) - s + 1 of them: s^(k-t) - 1 full groups, in each of which
+    # B_s adds the leading prefix to the other s - 1 entries, and one entry left over.  Summed over
+    # t = 1 .. k-1: (s-1) * sum_j (s^j - 1) = n - s - (k-1)(s-1).
+    n = s ** k
+    c_up, c_all = tm.Counters(s), tm.Counters(s)
+    tm.matmul_scan(np.ones(n, dtype=np.int64), s, c_up, up_sweep_only=True)
+    tm.matmul_scan(np.ones(n, dtype=np.int64), s, c_all)
+    assert c_up.useful_adds == s * (n - 1) // 2
+    assert c_all.useful_adds - c_up.useful_adds == n - s - (k - 1) * (s - 1)      # the B_s rounds alone, exactly
+    # a scan needs at least n - 1 additions, and the lemma's bound holds
+    assert n - 1 <= c_all.useful_adds <= math.ceil(n * (1 + s / 2)) + s ** 3 * k
+
+
+def test_constant_matrices_entry_by_entry():
+    for s in (2, 3, 5, 16):
+        L, Bm = tm.L_matrix(s), tm.B_matrix(s)
+        for i in range(s):
+            for j in range(s):
+                assert L[i, j] == (1 if j <= i else 0)
+                assert Bm[i, j] == (1 if (j == i or j == 0) else 0)
+
+
 @pytest.mark.parametrize("k", range(1, 11))
 def test_s2_work_equals_brent_kung(k):
     # Table 1: Brent-Kung performs 2n - log2(n) - 2 additions, and Algorithm 1 with s = 2 is Brent-Kung
