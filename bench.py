@@ -3,6 +3,8 @@
 
     python bench.py --gpus N --steps K --warmup W            # this library (CUDA, through the C ABI)
     python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
+    python bench.py --fixed-cost                             # where the microseconds of a small launch go
+    python bench.py --profile ...                            # the bare loop that is wrapped in ncu
 
 A step is one scan of the headline workload: n = 2^28 int8 values uniform in [-127, 127],
 int32 output, s = 16 (256 MiB read, 1 GiB written).  With N > 1 every rank scans its own
@@ -18,6 +20,7 @@ import statistics
 import subprocess
 import sys
 import tempfile
+import threading
 import time
 
 import numpy as np
@@ -30,9 +33,11 @@ N_ELEMS = 1 << 28
 S_TILE = 16
 BYTES_PER_ELEM = 5          # int8 read + int32 written
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the main kernel on 2^26 elements, from the
-# ncu capture summarised in profiles/ (traffic grows in proportion to n: one read and one write per element)
-NCU_TRAFFIC_BYTES_PER_2P26 = 278.2e6   # profiles/tcu_scan_kernel_int8_s16_n2p26_ncu_full.md; scaled by n / 2^26 below
+# From the ncu capture of the main kernel on 2^26 elements (profiles/tcu_scan_kernel_int8_s16_n2p26_ncu_full.md):
+# DRAM bytes read / input bytes, and bytes the SMs wrote to L2 / output bytes.  DRAM *write* bytes of a capture are
+# not used: tens of MB of the output are still dirty in L2 when the kernel ends, a constant that does not grow with n.
+NCU_READ_RATIO = 1.011
+NCU_WRITE_RATIO = 1.011
 
 
 def measured_peak():
@@ -42,6 +47,17 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
 
 class ClockSampler:
@@ -105,6 +121,35 @@ def oracle_leg(x: np.ndarray, reps: int):
     return x.size / best, y
 
 
+def oracle_all_cores(x: np.ndarray, threads: int):
+    """A second, separately labelled CPU figure: the same C loop of the oracle on every host core.  The array is
+    cut into one chunk per thread; pass 1 scans every chunk from zero to learn its total, pass 2 scans it again
+    starting from the sum of the chunks before it (the classical chunked two-pass scan; ctypes releases the GIL
+    inside the C loop, so Python threads do run side by side)."""
+    from oracle import scan_oracle as so
+    bounds = np.linspace(0, x.size, threads + 1).astype(np.int64)
+    totals = [0] * threads
+
+    def pass1(k):
+        totals[k] = int(so.scan_i8(x[bounds[k]:bounds[k + 1]])[-1]) if bounds[k + 1] > bounds[k] else 0
+
+    def pass2(k, carry):
+        so.scan_i8(x[bounds[k]:bounds[k + 1]], init=carry)
+
+    def run(fn, args):
+        ts = [threading.Thread(target=fn, args=a) for a in args]
+        for t in ts:
+            t.start()
+        for t in ts:
+            t.join()
+
+    t0 = time.perf_counter()
+    run(pass1, [(k,) for k in range(threads)])
+    carries = np.concatenate(([0], np.cumsum(totals)[:-1]))
+    run(pass2, [(k, int(carries[k])) for k in range(threads)])
+    return x.size / (time.perf_counter() - t0)
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -123,49 +168,131 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "elements/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "i64", "data": "synthetic",
-        "config": {"workload": "C3: inclusive scan, n=2^28 int8 uniform[-127,127] -> int32, s=16"},
+        "config": {"workload": "C3: inclusive scan, n=2^28 int8 uniform[-127,127] -> int32, s=16, one array per GPU"},
         "cpu_baseline": {"value": value, "unit": "elements/s", "cores": 1, "kind": "oracle",
-                         "sample": f"whole 2^28-element input per step, {args.steps} steps"},
+                         "sample": f"whole 2^28-element input per step, {args.steps} steps",
+                         "host_cores": os.cpu_count(), "cpu_model": cpu_model()},
         "e2e": {"value": value, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
 
 
-def time_extra(B, torch, name, x, rows, cols, dt, s, exclusive, ws_ptr, ws_bytes, reps=10, two_sweep=False):
+class Timer:
+    """CUDA-event timing of back-to-back launches on torch's current stream (the stream every call is given)."""
+
+    def __init__(self, torch):
+        self.torch = torch
+
+    def loop(self, call, reps):
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def each(self, call, reps):
+        """Every launch between its own pair of events: median and best in microseconds."""
+        torch = self.torch
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+        ev[0].record()
+        for i in range(reps):
+            call()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        us = [1e3 * ev[i].elapsed_time(ev[i + 1]) for i in range(reps)]
+        return statistics.median(us), min(us)
+
+
+def time_extra(B, torch, x, rows, cols, dt, s, ws_ptr, ws_bytes, reps=10, **options):
+    """One of the other workloads: microseconds per scan, GB/s of algorithmic traffic, and the call's statistics."""
     out = torch.empty(rows * cols, dtype=torch.int32 if dt == 0 else torch.float32, device="cuda")
     stream = torch.cuda.current_stream().cuda_stream
+    stats = {}
 
     def call():
-        if two_sweep:
-            B.check(B.tcu_scan_inclusive_twosweep(x, out, cols, dt, s, ws_ptr, ws_bytes, stream))
-        elif rows == 1:
-            fn = B.tcu_scan_exclusive if exclusive else B.tcu_scan_inclusive
-            B.check(fn(x, out, cols, dt, s, ws_ptr, ws_bytes, stream))
-        else:
-            B.check(B.tcu_scan_batched(x, out, rows, cols, dt, s, int(exclusive), ws_ptr, ws_bytes, stream))
+        B.check(B.tcu_scan_ex(x, out, rows, cols, dt, s, ws_ptr, ws_bytes, stream, stats=stats, **options))
     for _ in range(3):
         call()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        call()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
+    ms = Timer(torch).loop(call, reps)
     nbytes = rows * cols * ((1 if dt == 0 else 2) + 4)
     del out
-    st = B.tcu_scan_last_stats()
-    return {"workload": name, "ms": ms, "elements_per_s": rows * cols / (ms * 1e-3), "GB_per_s": nbytes / (ms * 1e-3) / 1e9,
-            "levels_used": st["levels_used"], "depth_bound_2floor_log_s_n": st["depth_bound"],
-            "sxs_products": st["sxs_products"], "n_over_s2": rows * cols // (s * s), "mma_instructions": st["mma_instructions"]}
+    return {"us": round(1e3 * ms, 2), "GBps": round(nbytes / (ms * 1e-3) / 1e9, 1)}, stats
+
+
+def fixed_cost(args):
+    """Takes the time of a small launch apart with the kernel's own time stamps (%globaltimer at fixed points,
+    written only when the caller passes a stamp buffer) and with host clocks around the call."""
+    import torch
+    from paper_2411_17887_b200 import binding as B
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream().cuda_stream
+    ws_bytes = B.tcu_scan_workspace_bytes(1, 1 << 26, 0, 16)
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+    ws_ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+    B.check(B.tcu_scan_workspace_init(ws_ptr, ws_bytes, stream))
+    g = torch.Generator(device="cuda").manual_seed(1)
+    xi = torch.randint(-127, 128, (1 << 26,), device="cuda", dtype=torch.int8, generator=g)
+    xf = (torch.rand(1 << 26, device="cuda", generator=g) * 2 - 1).half()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    stamps = torch.zeros(sms * B.TCU_SCAN_STAMPS_PER_CTA, dtype=torch.int64, device="cuda")
+    report = []
+    for name, x, n, dt in [("C1 n=2^16 int8", xi, 1 << 16, 0), ("C2 n=2^24 fp16", xf, 1 << 24, 1), ("C5 n=2^26 fp16", xf, 1 << 26, 1)]:
+        out = torch.empty(n, dtype=torch.int32 if dt == 0 else torch.float32, device="cuda")
+
+        def plain():
+            B.check(B.tcu_scan_inclusive(x, out, n, dt, 16, ws_ptr, ws_bytes, stream))
+
+        def stamped():
+            B.check(B.tcu_scan_ex(x, out, 1, n, dt, 16, ws_ptr, ws_bytes, stream, d_stamps=stamps))
+        for _ in range(5):
+            plain()
+        torch.cuda.synchronize()
+        t = Timer(torch)
+        back_to_back_us = 1e3 * t.loop(plain, 200)
+        med_us, best_us = t.each(plain, 200)
+        # host cost of one call (argument checks, tensor-map encoding, launch), the GPU kept busy so nothing blocks
+        t0 = time.perf_counter()
+        for _ in range(200):
+            plain()
+        host_us = 1e6 * (time.perf_counter() - t0) / 200
+        torch.cuda.synchronize()
+        # device-side stamps: isolated launches (stream idle before each), and a launch right behind another one
+        rows = {}
+        for mode in ("isolated", "behind_another"):
+            acc = []
+            for _ in range(20):
+                stamps.zero_()
+                torch.cuda.synchronize()
+                if mode == "behind_another":
+                    plain()
+                stamped()
+                torch.cuda.synchronize()
+                st = stamps.cpu().numpy().reshape(sms, B.TCU_SCAN_STAMPS_PER_CTA)
+                grid = min(sms, (n + 16383) // 16384)
+                st = st[:grid]
+                t_first = st[:, 0].min()
+                acc.append([float((st[:, k][st[:, k] > 0] - t_first).max()) / 1e3 if (st[:, k] > 0).any() else None
+                            for k in range(len(B.STAMP_NAMES))])
+            rows[mode] = {nm: round(statistics.median([a[k] for a in acc if a[k] is not None]), 2)
+                          for k, nm in enumerate(B.STAMP_NAMES) if any(a[k] is not None for a in acc)}
+        nbytes = n * ((1 if dt == 0 else 2) + 4)
+        report.append({"workload": name + ", s=16", "back_to_back_us": round(back_to_back_us, 2),
+                       "per_launch_us_median": round(med_us, 2), "per_launch_us_best": round(best_us, 2),
+                       "host_us_per_call": round(host_us, 2), "roofline_us_at_measured_peak": round(nbytes / measured_peak()[0] / 1e3, 2),
+                       "stamps_us_after_first_cta_entry_max_over_ctas": rows})
+        del out
+    print(json.dumps({"fixed_cost": report}))
 
 
 def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2411_17887_b200 import binding as B      # raises if the CUDA library is missing
-    from paper_2411_17887_b200 import inputs
+    from paper_2411_17887_b200 import inputs, sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -186,7 +313,8 @@ def run_ours(args):
     n = x_host.size
     d_in = torch.from_numpy(x_host).cuda()
     d_out = torch.empty(n, dtype=torch.int32, device="cuda")
-    ws_bytes = B.tcu_scan_workspace_bytes(4096, 1 << 28, 0, S_TILE)
+    ws_bytes = max(B.tcu_scan_workspace_bytes(4096, 65536, 0, S_TILE), B.tcu_scan_workspace_bytes(1, 1 << 28, 0, S_TILE),
+                   B.tcu_scan_segmented_workspace_bytes(1 << 28, 0, S_TILE))
     if args.profile:
         args.no_extras = True
     ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
@@ -199,15 +327,14 @@ def run_ours(args):
 
     if args.profile:
         # the loop that is wrapped in ncu: optionally another input type, tile size or variant of the upper levels
-        B.check(B.tcu_scan_set_upper_level_path(args.upper_level_path))
-        B.check(B.tcu_scan_set_down_sweep_path(args.down_sweep_path))
         if args.profile_dtype == "f16":
             d_in = torch.from_numpy(inputs.f16_uniform((n,), -1.0, 1.0, cfg.index)).cuda()
             d_out = torch.empty(n, dtype=torch.float32, device="cuda")
         prof_dt = B.DTYPES[args.profile_dtype]
 
         def step():  # noqa: F811
-            B.check(B.tcu_scan_inclusive(d_in, d_out, n, prof_dt, args.profile_s, ws_ptr, ws_bytes, stream))
+            B.check(B.tcu_scan_ex(d_in, d_out, 1, n, prof_dt, args.profile_s, ws_ptr, ws_bytes, stream,
+                                  upper_level_path=args.upper_level_path, down_sweep_path=args.down_sweep_path))
 
     # ---- device-resident timing
     for _ in range(max(args.warmup, 3)):
@@ -236,6 +363,9 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # every launch between its own events as well (outside the timed region above): median and best
+    launch_med_us, launch_best_us = Timer(torch).each(step, min(args.steps, 50))
+
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
     h_in = torch.from_numpy(x_host).pin_memory()
     h_out = torch.empty(n, dtype=torch.int32).pin_memory()
@@ -253,10 +383,9 @@ def run_ours(args):
     e2e_s = time.perf_counter() - t0
     clocks = sampler.stop() if sampler else None
 
-    times = torch.tensor([ms_total, e2e_s], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_s = float(times[0]), float(times[1])
+    # the slowest rank's times are the job's times
+    ms_total = sharding.max_over_ranks(ms_total, "cuda")
+    e2e_s = sharding.max_over_ranks(e2e_s, "cuda")
 
     if rank == 0:
         ms_step = ms_total / args.steps
@@ -270,9 +399,13 @@ def run_ours(args):
             "config": {"workload": f"C3: inclusive scan, n=2^{args.n_log2} int8 uniform[-127,127] -> int32, s=16, one array per GPU",
                        "n": n, "s": S_TILE, "l2": "working set 1.25 GiB per step, about 10x the L2, no flush needed",
                        "hbm_gb_per_s": achieved, "pct_of_8TBps": 100 * achieved / 8000.0,
-                       "pct_of_measured_copy": 100 * achieved / peak},
+                       "pct_of_measured_copy": 100 * achieved / peak,
+                       "launch_us_median": launch_med_us, "launch_us_best": launch_best_us},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES_PER_2P26 * n / (1 << 26), "peak_kind": f"of {peak_kind}",
+                         "traffic": n * (NCU_READ_RATIO * 1 + NCU_WRITE_RATIO * 4), "peak_kind": f"of {peak_kind}",
+                         "traffic_method": "algorithmic bytes x the ratios of an ncu capture at n=2^26 (DRAM read / input "
+                                           f"= {NCU_READ_RATIO}, SM-to-L2 write / output = {NCU_WRITE_RATIO}); DRAM write bytes of a "
+                                           "capture are not scaled: part of the output is still in L2 when the kernel ends",
                          "kernel": "tcu_scan_kernel<int8,s=16,inclusive>", "algorithmic_bytes_per_launch": BYTES_PER_ELEM * n},
             "e2e": {"value": world * n * e2e_steps / e2e_s, "unit": "elements/s", "h2d_bytes_per_step": n,
                     "d2h_bytes_per_step": 4 * n, "steps": e2e_steps, "ms_per_step": 1e3 * e2e_s / e2e_steps},
@@ -286,38 +419,64 @@ def run_ours(args):
             got = d_out.cpu().numpy()
             from oracle import scan_oracle as so
             rate, y = oracle_leg(x_host, 5)
-            line["cpu_baseline"] = {"value": rate, "unit": "elements/s", "cores": 1, "kind": "oracle",
-                                    "sample": f"whole 2^{args.n_log2}-element input, best of 5 sequential passes",
-                                    "host_cores": os.cpu_count()}
             line["parity"] = "bit-exact on all outputs" if np.array_equal(got, so.wrap_int32(y)) else "MISMATCH"
             del got, y
+            cores = os.cpu_count() or 1
+            line["cpu_baseline"] = {"value": rate, "unit": "elements/s", "cores": 1, "kind": "oracle",
+                                    "sample": f"whole 2^{args.n_log2}-element input, best of 5 sequential passes",
+                                    "host_cores": cores, "cpu_model": cpu_model(),
+                                    "all_cores": {"value": oracle_all_cores(x_host, cores), "unit": "elements/s", "threads": cores,
+                                                  "method": "the oracle's C loop on one chunk per thread, two passes "
+                                                            "(chunk totals, then every chunk rescanned from its carry)"}}
             if not args.no_extras:
-                extras = []
                 g = torch.Generator(device="cuda").manual_seed(inputs.BASE_SEED)
                 xf = (torch.rand(1 << 28, device="cuda", generator=g) * 2 - 1).half()
-                extras.append(time_extra(B, torch, "n=2^28 fp16 uniform[-1,1) -> fp32, s=16", xf, 1, 1 << 28, 1, 16, False, ws_ptr, ws_bytes))
-                extras.append(time_extra(B, torch, "C2: n=2^24 fp16, s=16, inclusive", xf, 1, 1 << 24, 1, 16, False, ws_ptr, ws_bytes))
-                extras.append(time_extra(B, torch, "C2: n=2^24 fp16, s=16, exclusive", xf, 1, 1 << 24, 1, 16, True, ws_ptr, ws_bytes))
+
+                def frac(r, nbytes=None):
+                    r["frac_of_peak"] = round(r["GBps"] / peak, 3)
+                    return r
+                # the second bandwidth target: fp16 -> fp32 at the headline size (kept in `config` so that it is
+                # part of the parsed line, not of the long tail)
+                r, _ = time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes)
+                line["config"]["fp16_n2p28_s16"] = dict(frac(r), pct_of_8TBps=round(100 * r["GBps"] / 8000.0, 1),
+                                                        elements_per_s=(1 << 28) / (r["us"] * 1e-6))
+                extra = {}
+                extra["C2_n2p24_f16_incl"] = frac(time_extra(B, torch, xf, 1, 1 << 24, 1, 16, ws_ptr, ws_bytes, reps=50)[0])
+                extra["C2_n2p24_f16_excl"] = frac(time_extra(B, torch, xf, 1, 1 << 24, 1, 16, ws_ptr, ws_bytes, reps=50, exclusive=1)[0])
                 for s in (16, 64, 128):
-                    extras.append(time_extra(B, torch, f"C5: n=2^26 fp16, s={s}", xf.abs(), 1, 1 << 26, 1, s, False, ws_ptr, ws_bytes))
+                    r, st = time_extra(B, torch, xf.abs(), 1, 1 << 26, 1, s, ws_ptr, ws_bytes, reps=20)
+                    extra[f"C5_n2p26_f16_s{s}"] = dict(frac(r), levels_used=st["levels_used"], depth_bound=st["depth_bound"],
+                                                       sxs_products=st["sxs_products"], mma=st["mma_instructions"])
                 xb = torch.randn(1 << 28, device="cuda", generator=g).bfloat16()
-                extras.append(time_extra(B, torch, "C4: 4096 x 65536 bf16 normal -> fp32, s=16, row-wise", xb, 4096, 65536, 2, 16, False, ws_ptr, ws_bytes))
-                extras.append(time_extra(B, torch, "C1: n=2^16 int8, s=16", d_in, 1, 1 << 16, 0, 16, False, ws_ptr, ws_bytes))
-                extras.append(time_extra(B, torch, "C3 in the two-sweep structure (reduce, scan totals, scan): n=2^28 int8, s=16",
-                                         d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes, two_sweep=True))
-                extras.append(time_extra(B, torch, "fp16 n=2^28 in the two-sweep structure, s=16",
-                                         xf, 1, 1 << 28, 1, 16, False, ws_ptr, ws_bytes, two_sweep=True))
-                # the same scan with the row-total level on tensor cores (8-bit limbs) instead of warp shuffles
-                B.check(B.tcu_scan_set_upper_level_path(1))
-                extras.append(time_extra(B, torch, "C3 with the scan over row totals as a tcgen05 product on 8-bit limbs (upper_level_path = 1)",
-                                         d_in, 1, n, 0, 16, False, ws_ptr, ws_bytes))
-                B.check(B.tcu_scan_set_upper_level_path(0))
+                extra["C4_4096x65536_bf16"] = frac(time_extra(B, torch, xb, 4096, 65536, 2, 16, ws_ptr, ws_bytes)[0])
+                del xb
+                extra["C1_n2p16_i8"] = time_extra(B, torch, d_in, 1, 1 << 16, 0, 16, ws_ptr, ws_bytes, reps=200)[0]
+                # the same scans in the two-sweep structure (reduce, scan the totals, scan with every carry known)
+                extra["C3_two_sweep"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, variant=1)[0])
+                extra["f16_n2p28_two_sweep"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, variant=1)[0])
+                # upper level (scan over the 128 row totals) as a tcgen05 product on exact narrow terms
+                extra["C3_upper_level_path1"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, upper_level_path=1)[0])
                 # fp16, s = 128: carries added by a tensor-core product (the paper's B_s step) instead of vector adds
                 for path in (0, 1):
-                    B.check(B.tcu_scan_set_down_sweep_path(path))
-                    extras.append(time_extra(B, torch, f"fp16 n=2^28, s=128, down_sweep_path = {path}", xf, 1, 1 << 28, 1, 128,
-                                             False, ws_ptr, ws_bytes))
-                B.check(B.tcu_scan_set_down_sweep_path(0))
+                    extra[f"f16_n2p28_s128_down_sweep_path{path}"] = frac(
+                        time_extra(B, torch, xf, 1, 1 << 28, 1, 128, ws_ptr, ws_bytes, down_sweep_path=path)[0])
+                del xf
+                # segmented scan of the headline array: random cut points, mean segment length 2^10, 2^14, 2^18
+                for logm in (10, 14, 18):
+                    cuts = torch.randint(0, n, (n >> logm,), device="cuda", generator=g, dtype=torch.int64)
+                    off = torch.cat([torch.zeros(1, dtype=torch.int64, device="cuda"), cuts.sort().values,
+                                     torch.full((1,), n, dtype=torch.int64, device="cuda")])
+                    seg_out = torch.empty(n, dtype=torch.int32, device="cuda")
+
+                    def seg_call():
+                        B.check(B.tcu_scan_segmented(d_in, seg_out, n, off, off.numel() - 1, 0, 16, 0, ws_ptr, ws_bytes, stream))
+                    for _ in range(2):
+                        seg_call()
+                    torch.cuda.synchronize()
+                    ms_seg = Timer(torch).loop(seg_call, 10)
+                    extra[f"segmented_n2p28_i8_mean2p{logm}"] = frac({"us": round(1e3 * ms_seg, 1),
+                                                                      "GBps": round(5 * n / (ms_seg * 1e-3) / 1e9, 1)})
+                    del seg_out, off, cuts
                 # application: radix sort of 2^24 keys by 32 one-bit splits, each an exclusive scan of int8 flags
                 ns = 1 << 24
                 keys = torch.randint(0, 1 << 31, (ns,), device="cuda", dtype=torch.int32, generator=g)
@@ -325,37 +484,25 @@ def run_ours(args):
                 tmp_bytes = B.tcu_sort_tmp_bytes(ns)
                 tmp = torch.empty(tmp_bytes + 256, dtype=torch.uint8, device="cuda")
                 tmp_ptr = tmp.data_ptr() + (-tmp.data_ptr()) % 256
+
+                def sort_call():
+                    B.check(B.tcu_sort_u32(keys, sorted_out, ns, tmp_ptr, tmp_bytes, ws_ptr, ws_bytes, stream))
                 for _ in range(2):
-                    B.check(B.tcu_sort_u32(keys, sorted_out, ns, tmp_ptr, tmp_bytes, ws_ptr, ws_bytes, stream))
+                    sort_call()
                 torch.cuda.synchronize()
-                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                s0.record()
-                for _ in range(3):
-                    B.check(B.tcu_sort_u32(keys, sorted_out, ns, tmp_ptr, tmp_bytes, ws_ptr, ws_bytes, stream))
-                s1.record()
-                torch.cuda.synchronize()
-                ms_sort = s0.elapsed_time(s1) / 3
-                ok = bool((sorted_out[1:] >= sorted_out[:-1]).all())
-                extras.append({"workload": "radix sort of 2^24 uint32 keys by 32 one-bit splits (32 exclusive scans)",
-                               "ms": ms_sort, "keys_per_s": ns / (ms_sort * 1e-3), "sorted": ok})
-                line["extra"] = extras
+                ms_sort = Timer(torch).loop(sort_call, 3)
+                extra["radix_sort_2p24_u32"] = {"us": round(1e3 * ms_sort, 1), "keys_per_s": ns / (ms_sort * 1e-3),
+                                                "sorted": bool((sorted_out[1:] >= sorted_out[:-1]).all())}
+                line["extra"] = extra
             if args.sweep_ctas:
                 sms = torch.cuda.get_device_properties(local).multi_processor_count
                 sweep = []
-                ps = [1, 2, 4, 8, 16, 32, 64, 128, sms]
-                for pcount in ps:
-                    B.check(B.tcu_scan_set_max_ctas(pcount))
-                    reps = 2 if pcount < 8 else 5
-                    step()
+                for pcount in [1, 2, 4, 8, 16, 32, 64, 128, sms]:
+                    def pstep():
+                        B.check(B.tcu_scan_ex(d_in, d_out, 1, n, B.TCU_I8_I32, S_TILE, ws_ptr, ws_bytes, stream, max_ctas=pcount))
+                    pstep()
                     torch.cuda.synchronize()
-                    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a0.record()
-                    for _ in range(reps):
-                        step()
-                    a1.record()
-                    torch.cuda.synchronize()
-                    sweep.append({"p": pcount, "ms": a0.elapsed_time(a1) / reps})
-                B.check(B.tcu_scan_set_max_ctas(0))
+                    sweep.append({"p": pcount, "ms": Timer(torch).loop(pstep, 2 if pcount < 8 else 5)})
                 t1 = sweep[0]["ms"]
                 for e in sweep:
                     e["speedup_vs_p1"] = t1 / e["ms"]
@@ -376,17 +523,21 @@ def main():
     ap.add_argument("--profile-dtype", default="i8", choices=["i8", "f16"], help="input type of the --profile loop")
     ap.add_argument("--profile-s", type=int, default=16, help="tile size s of the --profile loop")
     ap.add_argument("--upper-level-path", type=int, default=0, choices=[0, 1],
-                    help="1: scan the row totals with a tensor-core product on 8-bit limbs (int8 input)")
+                    help="--profile loop: 1 scans the row totals with a tensor-core product on exact narrow terms")
     ap.add_argument("--down-sweep-path", type=int, default=0, choices=[0, 1],
-                    help="1: add the row carries with a tensor-core product (fp16 input, s = 128)")
+                    help="--profile loop: 1 adds the row carries with a tensor-core product (fp16 input, s = 128)")
     ap.add_argument("--sweep-ctas", action="store_true",
                     help="also time the headline scan on p = 1, 2, 4, ... persistent CTAs (one per SM) and report time vs p")
     ap.add_argument("--n-log2", type=int, default=28, help="log2 of the array length (28 = the headline workload)")
     ap.add_argument("--profile", action="store_true",
                     help="device-resident loop only (no end-to-end leg, no oracle): the command to wrap in ncu")
+    ap.add_argument("--fixed-cost", action="store_true",
+                    help="break the time of small launches (C1, C2, C5) into phases with the kernel's time stamps")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.fixed_cost:
+        fixed_cost(args)
     else:
         run_ours(args)
 

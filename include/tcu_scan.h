@@ -15,8 +15,8 @@
  *    allocates or frees device memory and keeps no pointer after a call returns.
  *    Every `h_*` pointer is a HOST pointer.
  *  - All scan calls are asynchronous on `stream`.  Argument errors are detected on
- *    the host and returned before anything is launched.  A device-side wait that
- *    gave up (it never spins forever) is reported by tcu_scan_device_status().
+ *    the host and returned before anything is queued on the stream.  A device-side wait
+ *    that gave up (it never spins forever) is reported by tcu_scan_device_status().
  *  - Input and output must not overlap (element widths differ, so the paper's
  *    in-place form is not offered).  `d_in` and `d_out` must be 16-byte aligned.
  *  - Integer output is the exact sum modulo 2^32 (two's complement int32).
@@ -27,6 +27,11 @@
  *  - The workspace must have been cleared once by tcu_scan_workspace_init() before
  *    its first use; it may then be reused by any number of calls, of any shape whose
  *    requirement fits, as long as calls that share it do not overlap in time.
+ *  - The library keeps no state between calls except the bookkeeping of the calling
+ *    thread's last scan (tcu_scan_last_stats); every choice is an argument of the call.
+ *  - A "carry" that travels between calls (tcu_scan_options_t.d_carry_in / d_carry_out,
+ *    tcu_reduce_total, tcu_carry_exclusive_prefix) is an 8-byte device value: a double
+ *    for the floating-point types, a zero-extended uint32 for TCU_I8_I32.
  */
 #ifndef TCU_SCAN_H_
 #define TCU_SCAN_H_
@@ -59,13 +64,12 @@ typedef enum {
     TCU_BF16_F32 = 2 /* bf16  -> fp32         (tcgen05 kind::f16) */
 } tcu_dtype_t;
 
-/* What the last scan call of this process did (host-side bookkeeping, filled at launch). */
+/* What one scan call did (host-side bookkeeping, filled at launch). */
 typedef struct {
     uint64_t rows, cols;        /* problem shape (rows = 1 for the single-array calls)               */
     uint32_t s, dtype, exclusive;
     uint32_t variant;           /* 0 = single pass, decoupled look-back; 1 = two sweeps                 */
-    uint32_t upper_level_path;  /* 0 = levels above the products run on CUDA cores (warp shuffles);
-                                   1 = the scan over the 128 row totals is a tensor-core product on 8-bit limbs */
+    uint32_t upper_level_path;  /* where the levels above the U_s products ran: see tcu_scan_options_t */
     uint64_t tiles;             /* 128 x 128-element tiles processed                                  */
     uint64_t mma_instructions;  /* tcgen05.mma instructions issued                                    */
     uint64_t sxs_products;      /* s x s-equivalent U_s products they amount to ( = padded n / s^2 )  */
@@ -74,12 +78,55 @@ typedef struct {
     uint32_t depth_bound;       /* 2 floor(log_s cols), Corollary 1                                   */
     uint32_t grid, smem_bytes, in_stages, tail_elements;
     uint32_t down_sweep_path;   /* 0 = carries added on the vector ALUs; 1 = by a tensor-core product        */
+    uint32_t segments_path;     /* 0 = dense rows; 1 = segment boundaries inside the array (segmented call, or
+                                   batched rows whose length is not a multiple of 16)                    */
 } tcu_scan_stats_t;
+
+/* Per-call choices of tcu_scan_ex().  Zero-initialise, set struct_bytes = sizeof(tcu_scan_options_t),
+ * then set what differs from the defaults. */
+typedef struct {
+    uint32_t struct_bytes;
+    uint32_t exclusive;         /* 0 = inclusive, 1 = exclusive */
+    uint32_t variant;           /* 0 = single pass with decoupled look-back (default); 1 = two sweeps:
+                                   reduce every tile, scan the totals, then scan with every carry known
+                                   (reads the input twice; exists so that the choice can be measured)  */
+    uint32_t upper_level_path;  /* Paper Section 2 keeps every level of the up-sweep a product of two square
+                                   matrices; the totals that the upper levels work on are int32 / fp32,
+                                   which are not tensor-core input types.
+                                   0 (default) = upper levels on the CUDA cores (register chain along a
+                                       row, warp shuffles across the 128 rows of a tile);
+                                   1 = the scan over the 128 row totals of a tile is a tcgen05 product of
+                                       a strictly lower triangular all-ones matrix with the totals split
+                                       into exact narrow terms (two signed 8-bit limbs for int8 input,
+                                       three bf16 terms for fp16 / bf16 input), recombined afterwards.
+                                   Integer results are identical, floating-point results satisfy the
+                                   same tolerance. */
+    uint32_t down_sweep_path;   /* Paper Section 2, matrix B_s, and the discussion's remark that the tensor
+                                   unit is used at O(1/s) in the down-sweep.  1 = fp16 / bf16 scans with
+                                   s = 128 add each row's carry to the whole row by a tcgen05 product
+                                   (accumulator += C * ones, C holding the carry split exactly into three
+                                   bf16 terms) instead of one vector add per element; ignored otherwise. */
+    uint32_t max_ctas;          /* 0 = one persistent CTA per SM; otherwise at most this many.  One CTA owns
+                                   one SM's tensor core, so this is the p of the paper's p-TCU time bound
+                                   O(n(1 + l/s^2)/p + (s^2 + l) log_s n) (Section 2.2, last paragraph).
+                                   Results do not depend on it. */
+    const void *d_carry_in;     /* single array only: carry (8 bytes, see above) that precedes x[0], or NULL */
+    void *d_carry_out;          /* single array only: receives carry_in + x[0] + ... + x[n-1] (8 bytes), or NULL;
+                                   not written when n = 0 */
+    uint64_t *d_stamps;         /* NULL, or TCU_SCAN_STAMPS_PER_CTA values per CTA of the launch (at most one
+                                   CTA per SM): %globaltimer nanoseconds at fixed points of the kernel, for
+                                   taking the fixed cost of a launch apart (index meanings: entry, set-up
+                                   done, previous kernel done, first tile claimed, landed, published, carry
+                                   known, stored, role loops done, all warps done, exit, tiles by group 0/1) */
+} tcu_scan_options_t;
+#define TCU_SCAN_STAMPS_PER_CTA 16
 
 /* Bytes of device workspace needed to scan `rows` independent rows of `cols` elements
  * (rows = 1 for the single-array calls).  Holds the per-tile {flag, aggregate / inclusive
  * prefix} records of the cross-tile carry scan (Section 2.2 steps 2-3: segment totals and
- * their scan).  Never fails; returns a small non-zero size even for empty problems. */
+ * their scan); when cols is not a multiple of 16 and rows > 1, also the per-row boundary
+ * notes of the segmented path.  Never fails; returns a small non-zero size even for empty
+ * problems. */
 size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s);
 
 /* Clear a workspace (asynchronous memset on `stream`).  Must run once before the first
@@ -95,6 +142,45 @@ tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t s
 tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                 void *d_ws, size_t ws_bytes, cudaStream_t stream);
 
+/* Exclusive scan, y[0] = 0, y[i] = x[0] + ... + x[i-1]  (the paper names the exclusive
+ * form only in Table 1; this is the standard reading: shifted by one, identity 0 in front).
+ * Arguments as for tcu_scan_inclusive. */
+tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
+                                void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* `rows` independent scans of `cols` elements each, dense row-major (row stride = cols)
+ * (Section 2.2 step 1: the algorithm run on each contiguous segment, no stitching).
+ * Any cols >= 1.  When cols is a multiple of 16 every row starts 16-byte aligned and the rows
+ * are tiled one by one; otherwise the array is tiled as a whole and the row starts are
+ * segment boundaries inside it (the path of tcu_scan_segmented; rows * cols < 2^40).
+ *   d_ws   at least tcu_scan_workspace_bytes(rows, cols, dt, s) bytes */
+tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols,
+                              tcu_dtype_t dt, int s, int exclusive,
+                              void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Segmented scan: the array is cut into `num_segments` consecutive segments and every segment
+ * is scanned on its own (Section 2.2, steps 1-4, with the segments given by the caller instead
+ * of the base-s digits of n: scan each segment, take the segment totals, scan them, add them
+ * back - here with the chain of carries cut at every segment start).
+ *   d_offsets  device, num_segments + 1 values of uint64: segment k is [offsets[k], offsets[k+1]);
+ *              non-decreasing, offsets[0] = 0, offsets[num_segments] = n (the caller's promise:
+ *              the values live on the device and are not checked); empty segments are allowed
+ *   d_ws       at least tcu_scan_segmented_workspace_bytes(n, dt, s) bytes, cleared once like any
+ *              workspace
+ * Elements of a segment whose 128-element row (rows are counted from the start of the array)
+ * holds no segment start go through the tensor-core path; rows that hold a start are rescanned
+ * from that start on by CUDA cores. */
+size_t tcu_scan_segmented_workspace_bytes(size_t n, tcu_dtype_t dt, int s);
+tcu_status_t tcu_scan_segmented(const void *d_in, void *d_out, size_t n, const uint64_t *d_offsets,
+                                size_t num_segments, tcu_dtype_t dt, int s, int exclusive,
+                                void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* The general form: rows = 1 for a single array.  `opt` may be NULL (all defaults); `stats_out`
+ * may be NULL, otherwise it receives what tcu_scan_last_stats() would return after this call. */
+tcu_status_t tcu_scan_ex(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
+                         const tcu_scan_options_t *opt, tcu_scan_stats_t *stats_out,
+                         void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
 /* Inclusive scan for callers that cannot hand the library a workspace.  (The paper has no
  * counterpart for this entry point; it exists for integration reasons only.)
  *
@@ -106,7 +192,7 @@ tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dty
  * The caller still passes the input and the output; the call allocates and frees nothing.
  *
  *   n       at most TCU_SCAN_NOALLOC_MAX_ELEMENTS, else TCU_ERR_TOO_LARGE (nothing is launched)
- *   others  as for tcu_scan_inclusive
+ *   others  as for tcu_scan_inclusive; they are checked before anything is queued on the stream
  *
  * Cost: every GPU on which the library is loaded holds about 64 KiB for the array until the
  * process ends, whether this entry point is used or not.
@@ -115,34 +201,17 @@ tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dty
  * Sharing: there is one array per device and every call uses it, so two calls whose kernels
  * could overlap on the GPU (different streams, no dependency between them) corrupt each
  * other's carries; serialise them.  Each call clears the part of the array it needs, on
- * `stream`, before its kernel runs. */
+ * `stream`, before its kernel runs - which also wipes the record of an earlier time-out, so
+ * ask tcu_scan_noalloc_status() after a call whose result matters, before the next call. */
 #define TCU_SCAN_NOALLOC_MAX_ELEMENTS (1u << 26)
 tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                         cudaStream_t stream);
 
-/* Exclusive scan, y[0] = 0, y[i] = x[0] + ... + x[i-1]  (the paper names the exclusive
- * form only in Table 1; this is the standard reading: shifted by one, identity 0 in front).
- * Arguments as for tcu_scan_inclusive. */
-tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
-                                void *d_ws, size_t ws_bytes, cudaStream_t stream);
-
-/* The same inclusive scan in the two-sweep structure of classical work-efficient scans (the
- * paper's up-sweep / down-sweep split across kernels): sweep 1 reads the input and reduces every
- * tile to its total, a one-block kernel scans the totals, sweep 2 is the single-pass kernel with
- * every carry already known.  It reads the input twice and exists so that the choice between
- * the two structures can be measured; results satisfy the same parity bars.  Arguments as for
- * tcu_scan_inclusive. */
-tcu_status_t tcu_scan_inclusive_twosweep(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
-                                         void *d_ws, size_t ws_bytes, cudaStream_t stream);
-
-/* `rows` independent scans of `cols` elements each, dense row-major (row stride = cols)
- * (Section 2.2 step 1: the algorithm run on each contiguous segment, no stitching).
- * cols must be a multiple of 16 (so that every row starts 16-byte aligned in both arrays), else
- * TCU_ERR_UNSUPPORTED.
- *   d_ws   at least tcu_scan_workspace_bytes(rows, cols, dt, s) bytes */
-tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols,
-                              tcu_dtype_t dt, int s, int exclusive,
-                              void *d_ws, size_t ws_bytes, cudaStream_t stream);
+/* What tcu_scan_device_status() is for a workspace, for the built-in array of
+ * tcu_scan_inclusive_noalloc on the current device: synchronises `stream`, then returns TCU_OK,
+ * or TCU_ERR_TIMEOUT if the most recent noalloc call gave up a bounded wait.  (No counterpart
+ * in the paper.)  Allocates nothing. */
+tcu_status_t tcu_scan_noalloc_status(cudaStream_t stream);
 
 /* Debug / teaching entry: only up-sweep round t = 0 of Algorithm 1, i.e. every chunk of
  * s consecutive elements replaced by its own inclusive scan (W = L_s T), no carries.
@@ -153,8 +222,9 @@ tcu_status_t tcu_scan_level0_debug(const void *d_in, void *d_out, size_t n, tcu_
 /* Host-buffer form: uploads h_in to d_in, scans, downloads d_out to h_out.  Everything is
  * asynchronous; the caller synchronises `stream` before reading h_out (that also covers the
  * copies, which long inclusive scans run on two internal streams so that upload, scan and
- * download of successive 2^24-element pieces overlap; each piece continues from the last output
- * of the piece before it).  h_in / h_out should be pinned, otherwise the copies serialise.
+ * download of successive 2^24-element pieces overlap; each piece continues from the total of
+ * the pieces before it, handed over as an 8-byte carry inside the workspace).  h_in / h_out
+ * should be pinned, otherwise the copies serialise.
  * d_in / d_out are caller-owned device staging buffers of n input / n output elements; they and
  * the workspace are in use until `stream` has drained. */
 tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t dt, int s, int exclusive,
@@ -164,17 +234,38 @@ tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t 
  * `d_ws` since its last init gave up a bounded wait (its output is then not valid). */
 tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream);
 
-/* Self-test of the failure path (no counterpart in the paper): launches one warp that waits,
- * for at most `limit_ms` milliseconds (1..1000), on a tile record that nothing publishes, and
- * then records the time-out in the workspace header the way the scan kernels do.  After the
- * stream has drained, tcu_scan_device_status(d_ws) returns TCU_ERR_TIMEOUT and the context is
- * still usable; tcu_scan_workspace_init() clears the condition.  Nothing faults or hangs. */
-tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned limit_ms, cudaStream_t stream);
+/* Self-test of the failure path (no counterpart in the paper): runs the ordinary inclusive scan
+ * kernel on the given input, except that the records of tile `skip_tile` (128 x 128 elements per
+ * tile) are never published and every device-side wait gives up after `limit_ms` milliseconds
+ * (1..1000) instead of about a second.  Tiles after `skip_tile` therefore wait in vain, the
+ * kernel records the time-out, winds down (drains its copies, frees its tensor memory) and
+ * returns.  After the stream has drained, tcu_scan_device_status(d_ws) returns TCU_ERR_TIMEOUT,
+ * the output is not valid, and the context is still usable; tcu_scan_workspace_init() clears
+ * the condition.  Nothing faults or hangs.  skip_tile must be below the number of tiles, and
+ * n a multiple of 128. */
+tcu_status_t tcu_scan_selftest_timeout(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
+                                       size_t skip_tile, unsigned limit_ms,
+                                       void *d_ws, size_t ws_bytes, cudaStream_t stream);
+
+/* One array split over several devices (paper Section 2.2 steps 2-4 with one segment per device,
+ * and the p-TCU bound of its last paragraph): each device computes the total of its shard
+ * (tcu_reduce_total), the totals are exchanged by the caller (8 bytes per device, e.g. an NCCL
+ * all-gather into local memory), each device sums the totals of the shards before its own
+ * (tcu_carry_exclusive_prefix) and scans its shard with that carry (tcu_scan_ex, d_carry_in).
+ *
+ * tcu_reduce_total: *d_total = x[0] + ... + x[n-1] as an 8-byte carry.  d_in 16-byte aligned;
+ *   d_ws as for a scan of n elements (its tile records are used as scratch).
+ * tcu_carry_exclusive_prefix: *d_carry = totals[0] + ... + totals[index-1] (8-byte carries,
+ *   count >= index values at d_totals). */
+tcu_status_t tcu_reduce_total(const void *d_in, size_t n, tcu_dtype_t dt, void *d_total,
+                              void *d_ws, size_t ws_bytes, cudaStream_t stream);
+tcu_status_t tcu_carry_exclusive_prefix(const void *d_totals, size_t count, size_t index, tcu_dtype_t dt,
+                                        void *d_carry, cudaStream_t stream);
 
 /* Radix sort of 32-bit unsigned keys by 32 stable one-bit splits, each split an exclusive
- * tcu scan of int8 flags (the paper's introduction: with Blelloch's reduction of radix sort to
- * prefix sums, a tensor-core-unit machine can sort).  An application of the scan, not a tuned
- * sort.
+ * tcu scan of int8 flags (the paper's introduction asks whether a tensor-core-unit machine
+ * can sort; with Blelloch's reduction of radix sort to prefix sums it can).  An application
+ * of the scan, not a tuned sort.
  *   d_keys_in / d_keys_out   device, n keys each, 16-byte aligned, must not overlap
  *   d_tmp                    device scratch of tcu_sort_tmp_bytes(n) bytes, 256-byte aligned
  *   d_ws                     scan workspace of tcu_scan_workspace_bytes(1, n, TCU_I8_I32, 16) bytes
@@ -183,30 +274,7 @@ size_t tcu_sort_tmp_bytes(size_t n);
 tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_t n, void *d_tmp, size_t tmp_bytes,
                           void *d_ws, size_t ws_bytes, cudaStream_t stream);
 
-/* Experiment knob (paper Section 2: "all numerical operations are multiplications between two
- * square matrices"): path = 1 makes the following int8 scans of this process compute the scan over
- * the 128 row totals of a tile - an upper level of the up-sweep, whose int32 operands are not a
- * tensor-core input type - as a tcgen05 kind::i8 product of a strictly lower triangular all-ones
- * matrix with the totals split into two signed 8-bit limbs, recombined exactly.  path = 0 (default)
- * uses warp shuffles.  Results are identical; tcu_scan_stats_t.upper_level_path records the choice.
- * Floating-point inputs always use path 0. */
-tcu_status_t tcu_scan_set_upper_level_path(int path);
-
-/* Experiment knob (paper Section 2, matrix B_s, and the discussion's remark that the tensor unit is
- * used at O(1/s) in the down-sweep): path = 1 makes the following fp16 / bf16 scans with s = 128
- * add each row's carry to the whole row by a tcgen05 product - accumulator += C * ones, C holding
- * the carry split exactly into three bf16 terms - instead of one vector add per element.  Other
- * dtypes and tile sizes ignore it.  Results satisfy the same tolerance;
- * tcu_scan_stats_t.down_sweep_path records the choice. */
-tcu_status_t tcu_scan_set_down_sweep_path(int path);
-
-/* Experiment knob: run the following scans of this process on at most `max_ctas` persistent CTAs,
- * i.e. on that many SMs (0 restores the default, one CTA per SM).  One CTA owns one SM's tensor
- * core, so this is the p of the paper's p-TCU time bound O(n(1 + l/s^2)/p + (s^2 + l) log_s n)
- * (Section 2.2, last paragraph, and the abstract).  Results do not depend on it. */
-tcu_status_t tcu_scan_set_max_ctas(int max_ctas);
-
-/* Copies the bookkeeping of the most recent scan call made by this process. */
+/* Copies the bookkeeping of the most recent scan call made by the calling thread. */
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out);
 
 const char *tcu_status_string(tcu_status_t st);

@@ -31,7 +31,21 @@ class TcuScanStats(ctypes.Structure):
                 ("tiles", ctypes.c_uint64), ("mma_instructions", ctypes.c_uint64), ("sxs_products", ctypes.c_uint64),
                 ("levels_used", ctypes.c_uint32), ("depth_bound", ctypes.c_uint32),
                 ("grid", ctypes.c_uint32), ("smem_bytes", ctypes.c_uint32), ("in_stages", ctypes.c_uint32),
-                ("tail_elements", ctypes.c_uint32), ("down_sweep_path", ctypes.c_uint32)]
+                ("tail_elements", ctypes.c_uint32), ("down_sweep_path", ctypes.c_uint32),
+                ("segments_path", ctypes.c_uint32)]
+
+
+class TcuScanOptions(ctypes.Structure):
+    _fields_ = [("struct_bytes", ctypes.c_uint32), ("exclusive", ctypes.c_uint32), ("variant", ctypes.c_uint32),
+                ("upper_level_path", ctypes.c_uint32), ("down_sweep_path", ctypes.c_uint32),
+                ("max_ctas", ctypes.c_uint32), ("d_carry_in", ctypes.c_void_p), ("d_carry_out", ctypes.c_void_p),
+                ("d_stamps", ctypes.c_void_p)]
+
+
+TCU_SCAN_STAMPS_PER_CTA = 16
+STAMP_NAMES = ("entry", "setup_done", "previous_kernel_done", "first_tile_claimed", "first_tile_landed",
+               "first_total_published", "first_carry_known", "first_tile_stored", "role_loops_done",
+               "all_warps_done", "exit")
 
 
 _vp, _sz, _int = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
@@ -39,7 +53,7 @@ _lib.tcu_scan_workspace_bytes.argtypes = [_sz, _sz, _int, _int]
 _lib.tcu_scan_workspace_bytes.restype = _sz
 _lib.tcu_scan_workspace_init.argtypes = [_vp, _sz, _vp]
 _lib.tcu_scan_workspace_init.restype = _int
-for _name in ("tcu_scan_inclusive", "tcu_scan_exclusive", "tcu_scan_level0_debug", "tcu_scan_inclusive_twosweep"):
+for _name in ("tcu_scan_inclusive", "tcu_scan_exclusive", "tcu_scan_level0_debug"):
     getattr(_lib, _name).argtypes = [_vp, _vp, _sz, _int, _int, _vp, _sz, _vp]
     getattr(_lib, _name).restype = _int
 _lib.tcu_scan_inclusive_noalloc.argtypes = [_vp, _vp, _sz, _int, _int, _vp]
@@ -50,18 +64,25 @@ _lib.tcu_scan_host.argtypes = [_vp, _vp, _sz, _int, _int, _int, _vp, _vp, _vp, _
 _lib.tcu_scan_host.restype = _int
 _lib.tcu_scan_device_status.argtypes = [_vp, _vp]
 _lib.tcu_scan_device_status.restype = _int
-_lib.tcu_scan_selftest_timeout.argtypes = [_vp, _sz, ctypes.c_uint, _vp]
+_lib.tcu_scan_selftest_timeout.argtypes = [_vp, _vp, _sz, _int, _int, _sz, ctypes.c_uint, _vp, _sz, _vp]
 _lib.tcu_scan_selftest_timeout.restype = _int
+_lib.tcu_scan_noalloc_status.argtypes = [_vp]
+_lib.tcu_scan_noalloc_status.restype = _int
+_lib.tcu_scan_ex.argtypes = [_vp, _vp, _sz, _sz, _int, _int, ctypes.POINTER(TcuScanOptions), ctypes.POINTER(TcuScanStats),
+                             _vp, _sz, _vp]
+_lib.tcu_scan_ex.restype = _int
+_lib.tcu_scan_segmented_workspace_bytes.argtypes = [_sz, _int, _int]
+_lib.tcu_scan_segmented_workspace_bytes.restype = _sz
+_lib.tcu_scan_segmented.argtypes = [_vp, _vp, _sz, _vp, _sz, _int, _int, _int, _vp, _sz, _vp]
+_lib.tcu_scan_segmented.restype = _int
+_lib.tcu_reduce_total.argtypes = [_vp, _sz, _int, _vp, _vp, _sz, _vp]
+_lib.tcu_reduce_total.restype = _int
+_lib.tcu_carry_exclusive_prefix.argtypes = [_vp, _sz, _sz, _int, _vp, _vp]
+_lib.tcu_carry_exclusive_prefix.restype = _int
 _lib.tcu_sort_tmp_bytes.argtypes = [_sz]
 _lib.tcu_sort_tmp_bytes.restype = _sz
 _lib.tcu_sort_u32.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _sz, _vp]
 _lib.tcu_sort_u32.restype = _int
-_lib.tcu_scan_set_down_sweep_path.argtypes = [_int]
-_lib.tcu_scan_set_down_sweep_path.restype = _int
-_lib.tcu_scan_set_upper_level_path.argtypes = [_int]
-_lib.tcu_scan_set_upper_level_path.restype = _int
-_lib.tcu_scan_set_max_ctas.argtypes = [_int]
-_lib.tcu_scan_set_max_ctas.restype = _int
 _lib.tcu_scan_last_stats.argtypes = [ctypes.POINTER(TcuScanStats)]
 _lib.tcu_scan_last_stats.restype = _int
 _lib.tcu_status_string.argtypes = [_int]
@@ -99,8 +120,46 @@ def tcu_scan_inclusive_noalloc(d_in, d_out, n: int, dt: int, s: int, stream=0) -
     return _lib.tcu_scan_inclusive_noalloc(_p(d_in), _p(d_out), n, dt, s, stream)
 
 
-def tcu_scan_inclusive_twosweep(d_in, d_out, n: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0) -> int:
-    return _lib.tcu_scan_inclusive_twosweep(_p(d_in), _p(d_out), n, dt, s, _p(d_ws), ws_bytes, stream)
+def tcu_scan_noalloc_status(stream=0) -> int:
+    """TCU_OK, or TCU_ERR_TIMEOUT if the most recent noalloc call on this device gave up a wait (syncs `stream`)."""
+    return _lib.tcu_scan_noalloc_status(stream)
+
+
+def _stats_dict(st: TcuScanStats) -> dict:
+    return {name: int(getattr(st, name)) for name, _ in TcuScanStats._fields_}
+
+
+def tcu_scan_ex(d_in, d_out, rows: int, cols: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0, *,
+                exclusive: int = 0, variant: int = 0, upper_level_path: int = 0, down_sweep_path: int = 0,
+                max_ctas: int = 0, d_carry_in=None, d_carry_out=None, d_stamps=None, stats: dict = None) -> int:
+    """The general call: every per-call choice of ``tcu_scan_options_t`` as a keyword.  If ``stats`` is a dict
+    it is filled with the call's ``tcu_scan_stats_t``."""
+    opt = TcuScanOptions(ctypes.sizeof(TcuScanOptions), int(exclusive), int(variant), int(upper_level_path),
+                         int(down_sweep_path), int(max_ctas), _p(d_carry_in), _p(d_carry_out), _p(d_stamps))
+    st = TcuScanStats()
+    rc = _lib.tcu_scan_ex(_p(d_in), _p(d_out), rows, cols, dt, s, ctypes.byref(opt), ctypes.byref(st), _p(d_ws),
+                          ws_bytes, stream)
+    if stats is not None and rc == TCU_OK:
+        stats.update(_stats_dict(st))
+    return rc
+
+
+def tcu_scan_segmented_workspace_bytes(n: int, dt: int, s: int) -> int:
+    return int(_lib.tcu_scan_segmented_workspace_bytes(n, dt, s))
+
+
+def tcu_scan_segmented(d_in, d_out, n: int, d_offsets, num_segments: int, dt: int, s: int, exclusive: int, d_ws,
+                       ws_bytes: int, stream=0) -> int:
+    return _lib.tcu_scan_segmented(_p(d_in), _p(d_out), n, _p(d_offsets), num_segments, dt, s, int(exclusive),
+                                   _p(d_ws), ws_bytes, stream)
+
+
+def tcu_reduce_total(d_in, n: int, dt: int, d_total, d_ws, ws_bytes: int, stream=0) -> int:
+    return _lib.tcu_reduce_total(_p(d_in), n, dt, _p(d_total), _p(d_ws), ws_bytes, stream)
+
+
+def tcu_carry_exclusive_prefix(d_totals, count: int, index: int, dt: int, d_carry, stream=0) -> int:
+    return _lib.tcu_carry_exclusive_prefix(_p(d_totals), count, index, dt, _p(d_carry), stream)
 
 
 def tcu_scan_exclusive(d_in, d_out, n: int, dt: int, s: int, d_ws, ws_bytes: int, stream=0) -> int:
@@ -126,8 +185,10 @@ def tcu_scan_device_status(d_ws, stream=0) -> int:
     return _lib.tcu_scan_device_status(_p(d_ws), stream)
 
 
-def tcu_scan_selftest_timeout(d_ws, ws_bytes: int, limit_ms: int, stream=0) -> int:
-    return _lib.tcu_scan_selftest_timeout(_p(d_ws), ws_bytes, int(limit_ms), stream)
+def tcu_scan_selftest_timeout(d_in, d_out, n: int, dt: int, s: int, skip_tile: int, limit_ms: int, d_ws,
+                              ws_bytes: int, stream=0) -> int:
+    return _lib.tcu_scan_selftest_timeout(_p(d_in), _p(d_out), n, dt, s, int(skip_tile), int(limit_ms), _p(d_ws),
+                                          ws_bytes, stream)
 
 
 def tcu_sort_tmp_bytes(n: int) -> int:
@@ -138,24 +199,12 @@ def tcu_sort_u32(d_keys_in, d_keys_out, n: int, d_tmp, tmp_bytes: int, d_ws, ws_
     return _lib.tcu_sort_u32(_p(d_keys_in), _p(d_keys_out), n, _p(d_tmp), tmp_bytes, _p(d_ws), ws_bytes, stream)
 
 
-def tcu_scan_set_down_sweep_path(path: int) -> int:
-    return _lib.tcu_scan_set_down_sweep_path(int(path))
-
-
-def tcu_scan_set_upper_level_path(path: int) -> int:
-    return _lib.tcu_scan_set_upper_level_path(int(path))
-
-
-def tcu_scan_set_max_ctas(max_ctas: int) -> int:
-    return _lib.tcu_scan_set_max_ctas(int(max_ctas))
-
-
 def tcu_scan_last_stats() -> dict:
     st = TcuScanStats()
     rc = _lib.tcu_scan_last_stats(ctypes.byref(st))
     if rc != TCU_OK:
         raise RuntimeError(tcu_status_string(rc))
-    return {name: int(getattr(st, name)) for name, _ in TcuScanStats._fields_}
+    return _stats_dict(st)
 
 
 def check(rc: int) -> None:

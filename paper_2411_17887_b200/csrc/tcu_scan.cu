@@ -33,12 +33,9 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-std::atomic<int> g_upper_path{0};  // 0 = row totals scanned with warp shuffles, 1 = with a product on 8-bit limbs (int8 input only)
-std::atomic<int> g_down_path{0};   // 0 = carries added on the vector ALUs, 1 = by a tensor-core product (16-bit input, s = 128 only)
-std::atomic<int> g_max_ctas{0};   // 0 = one CTA per SM; otherwise the persistent grid is capped (scaling experiments)
-std::mutex g_stats_mutex;
-tcu_scan_stats_t g_stats;
-bool g_have_stats = false;
+// bookkeeping of the calling thread's most recent scan (nothing else outlives a call)
+thread_local tcu_scan_stats_t t_stats;
+thread_local bool t_have_stats = false;
 
 int elem_bytes(tcu_dtype_t dt) { return dt == TCU_I8_I32 ? 1 : 2; }
 bool valid_dtype(int dt) { return dt == TCU_I8_I32 || dt == TCU_F16_F32 || dt == TCU_BF16_F32; }
@@ -76,7 +73,6 @@ cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStrea
         if (e != cudaSuccess) return e;
         configured.store(dev);
     }
-#if TCU_PDL
     // programmatic dependent launch: this kernel's set-up (barriers, TMEM, constant operands) may overlap the
     // tail of whatever runs before it in the stream; it waits (griddepcontrol.wait) before touching global memory
     cudaLaunchConfig_t cfg = {};
@@ -90,10 +86,6 @@ cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStrea
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, tcu_scan_kernel<IS_INT, S, EXCL>, prm);
-#else
-    tcu_scan_kernel<IS_INT, S, EXCL><<<grid, kThreads, smem, stream>>>(prm);
-    return cudaGetLastError();
-#endif
 }
 
 template <bool IS_INT, bool EXCL>
@@ -121,38 +113,96 @@ bool overlaps(const void *a, size_t an, const void *b, size_t bn) {
     return pa < pb + bn && pb < pa + an;
 }
 
-tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
-                       bool exclusive, bool level0, void *d_ws, size_t ws_bytes, cudaStream_t stream,
-                       bool two_sweep = false, const void *d_carry_in = nullptr) {
-    if (!valid_dtype(dt) || !valid_s(s)) return (s > 0 && valid_dtype(dt)) ? TCU_ERR_UNSUPPORTED : TCU_ERR_INVALID_ARG;
-    if (rows == 0 || cols == 0) return TCU_OK;
-    if (!d_in || !d_out) return TCU_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(d_in) & 15) || (reinterpret_cast<uintptr_t>(d_out) & 15)) return TCU_ERR_INVALID_ARG;
+// Everything one scan launch needs to know.
+struct Call {
+    const void *d_in = nullptr;
+    void *d_out = nullptr;
+    size_t rows = 1, cols = 0;
+    tcu_dtype_t dt = TCU_I8_I32;
+    int s = 16;
+    bool exclusive = false, level0 = false, two_sweep = false;
+    int upper_path = 0, down_path = 0, max_ctas = 0;
+    const void *d_carry_in = nullptr;
+    void *d_carry_out = nullptr;
+    unsigned long long *d_stamps = nullptr;
+    long long spin_limit = kSpinLimitCycles;
+    uint32_t skip_tile = kNoTile;
+    void *d_ws = nullptr;
+    size_t ws_bytes = 0;
+    cudaStream_t stream = nullptr;
+    tcu_scan_stats_t *stats_out = nullptr;
+    // segmented scan (rows == 1): segment starts inside the array, either listed on the device or every seg_pitch elements
+    bool segmented = false;
+    const uint64_t *d_offsets = nullptr;
+    uint64_t seg_pitch = 0, num_segments = 0;
+};
+
+size_t round_up(size_t v, size_t to) { return (v + to - 1) / to * to; }
+size_t record_bytes(uint64_t tiles) { return size_t(kHeaderBytes) + 16 * size_t(tiles) + 16; }
+// workspace of a segmented scan of n elements: tile records, then one flag byte and one 4-byte value per row of 128
+size_t seg_flag_offset(uint64_t n) { return round_up(record_bytes(tiles_for(1, n)), 256); }
+size_t seg_val_offset(uint64_t n) { return seg_flag_offset(n) + round_up(size_t(n / kTileCols) + 1, 256); }
+size_t seg_workspace_bytes(uint64_t n) { return seg_val_offset(n) + 4 * (size_t(n / kTileCols) + 1); }
+size_t needed_workspace(const Call &c) {
+    return c.segmented ? seg_workspace_bytes(uint64_t(c.rows) * c.cols) : record_bytes(tiles_for(c.rows, c.cols));
+}
+
+// Host-side checks of a call; nothing has been queued on the stream when this returns an error.
+tcu_status_t check_call(const Call &c) {
+    if (!valid_dtype(c.dt) || !valid_s(c.s)) return (c.s > 0 && valid_dtype(c.dt)) ? TCU_ERR_UNSUPPORTED : TCU_ERR_INVALID_ARG;
+    if (c.rows == 0 || c.cols == 0) return TCU_OK;
+    if (!c.d_in || !c.d_out) return TCU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(c.d_in) & 15) || (reinterpret_cast<uintptr_t>(c.d_out) & 15)) return TCU_ERR_INVALID_ARG;
+    const int eb = elem_bytes(c.dt);
+    // dense rows: the row pitch must keep every row 16-byte aligned on both sides (TMA boxes, vector stores)
+    if (c.rows > 1 && ((c.cols * eb) % 16 != 0 || (c.cols * 4) % 16 != 0)) return TCU_ERR_UNSUPPORTED;
+    if (c.level0 && (c.cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
+    if (c.rows > (1ull << 31) || c.cols > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
+    if (c.rows > 1 && (c.d_carry_in || c.d_carry_out)) return TCU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(c.d_carry_in) & 7) || (reinterpret_cast<uintptr_t>(c.d_carry_out) & 7)) return TCU_ERR_INVALID_ARG;
+    if (c.two_sweep && (c.rows > 1 || c.d_carry_in || c.d_carry_out)) return TCU_ERR_UNSUPPORTED;
+    const uint64_t total = uint64_t(c.rows) * c.cols;
+    if (overlaps(c.d_in, total * eb, c.d_out, total * 4)) return TCU_ERR_INVALID_ARG;
+    if (!c.d_ws) return TCU_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(c.d_ws) & 255) return TCU_ERR_INVALID_ARG;
+    if (c.ws_bytes < needed_workspace(c)) return TCU_ERR_WORKSPACE;
+    if (c.segmented) {
+        if (c.rows != 1 || c.level0 || c.two_sweep || c.d_carry_in || c.d_carry_out) return TCU_ERR_UNSUPPORTED;
+        if (c.num_segments == 0 || c.num_segments > (1ull << 34)) return TCU_ERR_INVALID_ARG;
+        if (!c.d_offsets && c.seg_pitch == 0) return TCU_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(c.d_offsets) & 7) return TCU_ERR_INVALID_ARG;
+    }
+    const uint64_t tiles = tiles_for(c.rows, c.cols);
+    if (tiles >= (1ull << 31)) return TCU_ERR_UNSUPPORTED;
+    if (c.max_ctas < 0 || c.upper_path < 0 || c.upper_path > 1 || c.down_path < 0 || c.down_path > 1) return TCU_ERR_INVALID_ARG;
+    return TCU_OK;
+}
+
+tcu_status_t scan_impl(const Call &c) {
+    const tcu_status_t chk = check_call(c);
+    if (chk != TCU_OK || c.rows == 0 || c.cols == 0) return chk;
+    const void *d_in = c.d_in;
+    void *d_out = c.d_out;
+    const size_t rows = c.rows, cols = c.cols;
+    const tcu_dtype_t dt = c.dt;
+    const int s = c.s;
+    const bool exclusive = c.exclusive, level0 = c.level0, two_sweep = c.two_sweep;
+    void *d_ws = c.d_ws;
+    cudaStream_t stream = c.stream;
     const int eb = elem_bytes(dt);
-    // batched rows: the row pitch must keep every row 16-byte aligned on both sides (TMA boxes, vector stores)
-    if (rows > 1 && ((cols * eb) % 16 != 0 || (cols * 4) % 16 != 0)) return TCU_ERR_UNSUPPORTED;
-    if (level0 && (cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
-    if (rows > (1ull << 31) || cols > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
-    const uint64_t total = uint64_t(rows) * cols;
-    if (overlaps(d_in, total * eb, d_out, total * 4)) return TCU_ERR_INVALID_ARG;
-    if (!d_ws) return TCU_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
-    if (ws_bytes < tcu_scan_workspace_bytes(rows, cols, dt, s)) return TCU_ERR_WORKSPACE;
 
     const uint64_t rows128 = cols / kTileCols;
     const uint64_t tiles_per_row = (rows128 + kTileRows - 1) / kTileRows;
     const uint64_t tiles = rows * tiles_per_row;
     const uint32_t tail = uint32_t(cols % kTileCols);
-    if (tiles >= (1ull << 31)) return TCU_ERR_UNSUPPORTED;
-
     const int per32 = 32 / eb;
     const int seff = s > per32 ? s : per32;
     const int b_atoms = (seff * eb + 127) / 128;
     const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
     const uint32_t stage_bytes = kTileElems * eb;
-    const bool upper_tc = (dt == TCU_I8_I32) && g_upper_path.load() == 1;
-    const bool down_tc = (dt != TCU_I8_I32) && s == 128 && !level0 && g_down_path.load() == 1;
-    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? kUpperBytes : 0) +
+    const bool upper_tc = c.upper_path == 1 && !c.segmented && !level0;
+    const bool down_tc = (dt != TCU_I8_I32) && s == 128 && !level0 && c.down_path == 1 && !c.segmented;
+    const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? (dt == TCU_I8_I32 ? kUpperBytesInt : kUpperBytesFloat) : 0) +
                          (down_tc ? kDownBytes : 0) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kUseInStages) in_stages = kUseInStages;
@@ -170,7 +220,7 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     st.upper_level_path = upper_tc ? 1 : 0;
     st.down_sweep_path = down_tc ? 1 : 0;
     st.tiles = tiles;
-    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? 4 : 0) + (down_tc ? 1 : 0));  // U_s products + row-total products
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? (dt == TCU_I8_I32 ? 4 : 8) : 0) + (down_tc ? 1 : 0));  // U_s products + row-total products
     st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
     // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
     // scan over the tiles (absent for a single tile), carry add
@@ -179,6 +229,26 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
     st.in_stages = in_stages;
     st.smem_bytes = uint32_t(smem);
     st.tail_elements = tail;
+    st.segments_path = c.segmented ? 1 : 0;
+
+    // segmented scan: note, for every row of 128 elements that holds a segment start, whether it starts the row
+    // and what the row hands on (one warp per start), before the tile kernel runs
+    uint8_t *seg_flag = nullptr;
+    uint32_t *seg_val = nullptr;
+    SegSource seg{c.d_offsets, c.seg_pitch, c.num_segments};
+    const unsigned seg_blocks = unsigned((c.num_segments * 32 + 255) / 256);
+    if (c.segmented) {
+        seg_flag = reinterpret_cast<uint8_t *>(d_ws) + seg_flag_offset(cols);
+        seg_val = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_ws) + seg_val_offset(cols));
+        if (rows128 > 0) {
+            if (cudaMemsetAsync(seg_flag, 0, size_t(rows128), stream) != cudaSuccess) return TCU_ERR_CUDA;
+            if (dt == TCU_I8_I32)
+                tcu_segment_rows_kernel<true, false, kSegPrepare><<<seg_blocks, 256, 0, stream>>>(d_in, d_out, cols, seg, d_ws, uint32_t(tiles), seg_flag, seg_val, dt);
+            else
+                tcu_segment_rows_kernel<false, false, kSegPrepare><<<seg_blocks, 256, 0, stream>>>(d_in, d_out, cols, seg, d_ws, uint32_t(tiles), seg_flag, seg_val, dt);
+            if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+        }
+    }
 
     if (tiles > 0) {
         EncodeTiledFn encode = get_encode_fn();
@@ -187,6 +257,12 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
         if (sms <= 0) return TCU_ERR_CUDA;
         ScanParams prm;
         std::memset(&prm, 0, sizeof(prm));
+        // persistent grid: every CTA must be resident at once (the carry chain waits on
+        // lower-numbered tiles), so never more CTAs than SMs; one CTA fills an SM's shared memory
+        uint64_t ctas = uint64_t(sms);
+        const int cap = c.max_ctas;
+        if (cap > 0 && uint64_t(cap) < ctas) ctas = uint64_t(cap);
+
         const cuuint64_t dims[3] = {cuuint64_t(kTileCols), cuuint64_t(rows128), cuuint64_t(rows)};
         const cuuint32_t estr[3] = {1, 1, 1};
         // stride between scans: the row pitch for batched input; for a single array any multiple of
@@ -203,18 +279,15 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
         }
-        {
-            const cuuint64_t strides[2] = {cuuint64_t(kTileCols) * 4, pitch_elems * 4};
-            const cuuint32_t box[3] = {32, 32, 1};   // one slab: 32 columns x 32 rows, stored by one warp
-            CUtensorMapDataType ty = dt == TCU_I8_I32 ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-            CUresult r = encode(&prm.tmap_out, ty, 3, d_out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-            if (r != CUDA_SUCCESS) return TCU_ERR_CUDA;
-        }
         prm.ws = d_ws;
         prm.out = d_out;
-        prm.carry_in = (rows == 1 && !two_sweep) ? d_carry_in : nullptr;
+        prm.carry_in = c.d_carry_in;
+        prm.carry_out = c.d_carry_out;
+        prm.stamps = c.d_stamps;
+        prm.spin_limit = c.spin_limit;
+        prm.skip_publish_tile = c.skip_tile;
+        prm.seg_rowflag = seg_flag;
+        prm.seg_rowval = seg_val;
         prm.scan_pitch = cols;
         prm.rows128 = uint32_t(rows128);
         prm.tiles_total = uint32_t(tiles);
@@ -238,11 +311,6 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
             }
             if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
         }
-        // persistent grid: every CTA must be resident at once (the carry chain waits on
-        // lower-numbered tiles), so never more CTAs than SMs; one CTA fills an SM's shared memory
-        uint64_t ctas = uint64_t(sms);
-        const int cap = g_max_ctas.load();
-        if (cap > 0 && uint64_t(cap) < ctas) ctas = uint64_t(cap);
         dim3 grid(unsigned(tiles < ctas ? tiles : ctas));
         st.grid = grid.x;
         cudaError_t e;
@@ -252,23 +320,54 @@ tcu_status_t scan_impl(const void *d_in, void *d_out, size_t rows, size_t cols, 
             e = exclusive ? dispatch_s<false, true>(s, prm, grid, smem, stream) : dispatch_s<false, false>(s, prm, grid, smem, stream);
         if (e != cudaSuccess) return TCU_ERR_CUDA;
     }
-    if (tail > 0) {   // the last cols % 128 elements of every scan
+    if (c.segmented) {
+        // rows that hold a start: rescan them from the first start on; then the incomplete last row, if any
+        auto launch = [&](auto is_int, auto excl) {
+            constexpr bool I = decltype(is_int)::value, E = decltype(excl)::value;
+            if (rows128 > 0)
+                tcu_segment_rows_kernel<I, E, kSegFixup><<<seg_blocks, 256, 0, stream>>>(d_in, d_out, cols, seg, d_ws, uint32_t(tiles), seg_flag, seg_val, dt);
+            if (tail > 0)
+                tcu_segment_rows_kernel<I, E, kSegTail><<<1, 32, 0, stream>>>(d_in, d_out, cols, seg, d_ws, uint32_t(tiles), seg_flag, seg_val, dt);
+        };
+        if (dt == TCU_I8_I32) {
+            if (exclusive) launch(std::true_type{}, std::true_type{});
+            else launch(std::true_type{}, std::false_type{});
+        } else {
+            if (exclusive) launch(std::false_type{}, std::true_type{});
+            else launch(std::false_type{}, std::false_type{});
+        }
+        if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+    } else if (tail > 0) {   // the last cols % 128 elements of every scan
         const size_t start = size_t(rows128) * kTileCols;
         if (dt == TCU_I8_I32) {
-            if (exclusive) tcu_scan_tail_kernel<true, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
-            else tcu_scan_tail_kernel<true, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
+            if (exclusive) tcu_scan_tail_kernel<true, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, c.d_carry_in, c.d_carry_out);
+            else tcu_scan_tail_kernel<true, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, c.d_carry_in, c.d_carry_out);
         } else {
-            if (exclusive) tcu_scan_tail_kernel<false, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
-            else tcu_scan_tail_kernel<false, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, rows == 1 ? d_carry_in : nullptr);
+            if (exclusive) tcu_scan_tail_kernel<false, true><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, c.d_carry_in, c.d_carry_out);
+            else tcu_scan_tail_kernel<false, false><<<unsigned(rows), 128, 0, stream>>>(d_in, d_out, start, size_t(cols), tail, d_ws, uint32_t(tiles_per_row), dt, c.d_carry_in, c.d_carry_out);
         }
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
     }
-    {
-        std::lock_guard<std::mutex> lk(g_stats_mutex);
-        g_stats = st;
-        g_have_stats = true;
-    }
+    t_stats = st;
+    t_have_stats = true;
+    if (c.stats_out) *c.stats_out = st;
     return TCU_OK;
+}
+
+Call make_call(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s, bool exclusive, void *d_ws,
+               size_t ws_bytes, cudaStream_t stream) {
+    Call c;
+    c.d_in = d_in;
+    c.d_out = d_out;
+    c.rows = rows;
+    c.cols = cols;
+    c.dt = dt;
+    c.s = s;
+    c.exclusive = exclusive;
+    c.d_ws = d_ws;
+    c.ws_bytes = ws_bytes;
+    c.stream = stream;
+    return c;
 }
 
 // Built-in scratch of tcu_scan_inclusive_noalloc: the tile records of the cross-tile carry scan for
@@ -334,7 +433,8 @@ extern "C" {
 size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s) {
     (void)dt;
     (void)s;
-    return size_t(kHeaderBytes) + 16 * size_t(tiles_for(rows, cols)) + 16;
+    if (rows > 1 && cols % 16 != 0) return seg_workspace_bytes(uint64_t(rows) * cols);   // rows become segments of one array
+    return record_bytes(tiles_for(rows, cols));
 }
 
 tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t stream) {
@@ -345,13 +445,79 @@ tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t s
 
 tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
                                 size_t ws_bytes, cudaStream_t stream) {
-    return scan_impl(d_in, d_out, 1, n, dt, s, false, false, d_ws, ws_bytes, stream);
+    return scan_impl(make_call(d_in, d_out, 1, n, dt, s, false, d_ws, ws_bytes, stream));
+}
+
+tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
+                                size_t ws_bytes, cudaStream_t stream) {
+    return scan_impl(make_call(d_in, d_out, 1, n, dt, s, true, d_ws, ws_bytes, stream));
+}
+
+tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
+                              int exclusive, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    if (rows > 1 && cols % 16 != 0) {
+        // rows that do not start 16-byte aligned cannot be tiled one by one: tile the array as a whole and treat
+        // the row starts as segment starts
+        if (cols > (1ull << 40) / rows) return TCU_ERR_UNSUPPORTED;
+        Call c = make_call(d_in, d_out, 1, rows * cols, dt, s, exclusive != 0, d_ws, ws_bytes, stream);
+        c.segmented = true;
+        c.seg_pitch = cols;
+        c.num_segments = rows;
+        const tcu_status_t st = scan_impl(c);
+        if (st == TCU_OK) {          // report the shape the caller asked for
+            t_stats.rows = rows;
+            t_stats.cols = cols;
+        }
+        return st;
+    }
+    return scan_impl(make_call(d_in, d_out, rows, cols, dt, s, exclusive != 0, d_ws, ws_bytes, stream));
+}
+
+size_t tcu_scan_segmented_workspace_bytes(size_t n, tcu_dtype_t dt, int s) {
+    (void)dt;
+    (void)s;
+    return seg_workspace_bytes(n);
+}
+
+tcu_status_t tcu_scan_segmented(const void *d_in, void *d_out, size_t n, const uint64_t *d_offsets, size_t num_segments,
+                                tcu_dtype_t dt, int s, int exclusive, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+    if (n > 0 && (num_segments == 0 || !d_offsets)) return TCU_ERR_INVALID_ARG;
+    Call c = make_call(d_in, d_out, 1, n, dt, s, exclusive != 0, d_ws, ws_bytes, stream);
+    c.segmented = true;
+    c.d_offsets = d_offsets;
+    c.num_segments = num_segments;
+    return scan_impl(c);
+}
+
+tcu_status_t tcu_scan_ex(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
+                         const tcu_scan_options_t *opt, tcu_scan_stats_t *stats_out, void *d_ws, size_t ws_bytes,
+                         cudaStream_t stream) {
+    Call c = make_call(d_in, d_out, rows, cols, dt, s, false, d_ws, ws_bytes, stream);
+    c.stats_out = stats_out;
+    if (opt) {
+        if (opt->struct_bytes != sizeof(tcu_scan_options_t)) return TCU_ERR_INVALID_ARG;
+        if (opt->variant > 1 || opt->max_ctas > (1u << 20)) return TCU_ERR_INVALID_ARG;
+        if (opt->upper_level_path > 1 || opt->down_sweep_path > 1) return TCU_ERR_INVALID_ARG;
+        c.exclusive = opt->exclusive != 0;
+        c.two_sweep = opt->variant == 1;
+        c.upper_path = int(opt->upper_level_path);
+        c.down_path = int(opt->down_sweep_path);
+        c.max_ctas = int(opt->max_ctas);
+        c.d_carry_in = opt->d_carry_in;
+        c.d_carry_out = opt->d_carry_out;
+        c.d_stamps = reinterpret_cast<unsigned long long *>(opt->d_stamps);
+    }
+    return scan_impl(c);
 }
 
 tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                         cudaStream_t stream) {
     if (n > size_t(TCU_SCAN_NOALLOC_MAX_ELEMENTS)) return TCU_ERR_TOO_LARGE;
-    if (n == 0) return TCU_OK;
+    // every argument is checked before anything is queued on the stream (the scratch pointer is filled in below;
+    // a placeholder with the right alignment stands in for it during the check)
+    Call c = make_call(d_in, d_out, 1, n, dt, s, false, reinterpret_cast<void *>(uintptr_t(256)), kNoAllocScratchBytes, stream);
+    const tcu_status_t chk = check_call(c);
+    if (chk != TCU_OK || n == 0) return chk;
     void *scratch = nullptr;
     tcu_status_t st = noalloc_scratch(&scratch);
     if (st != TCU_OK) return st;
@@ -359,27 +525,22 @@ tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n,
     // expect to find at zero (header counters, the records of this call's tiles) is cleared here.
     const size_t used = tcu_scan_workspace_bytes(1, n, dt, s);
     if (cudaMemsetAsync(scratch, 0, used, stream) != cudaSuccess) return TCU_ERR_CUDA;
-    return scan_impl(d_in, d_out, 1, n, dt, s, false, false, scratch, kNoAllocScratchBytes, stream);
+    c.d_ws = scratch;
+    return scan_impl(c);
 }
 
-tcu_status_t tcu_scan_inclusive_twosweep(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
-                                         size_t ws_bytes, cudaStream_t stream) {
-    return scan_impl(d_in, d_out, 1, n, dt, s, false, false, d_ws, ws_bytes, stream, true);
-}
-
-tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
-                                size_t ws_bytes, cudaStream_t stream) {
-    return scan_impl(d_in, d_out, 1, n, dt, s, true, false, d_ws, ws_bytes, stream);
-}
-
-tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s,
-                              int exclusive, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
-    return scan_impl(d_in, d_out, rows, cols, dt, s, exclusive != 0, false, d_ws, ws_bytes, stream);
+tcu_status_t tcu_scan_noalloc_status(cudaStream_t stream) {
+    void *scratch = nullptr;
+    tcu_status_t st = noalloc_scratch(&scratch);
+    if (st != TCU_OK) return st;
+    return tcu_scan_device_status(scratch, stream);
 }
 
 tcu_status_t tcu_scan_level0_debug(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, void *d_ws,
                                    size_t ws_bytes, cudaStream_t stream) {
-    return scan_impl(d_in, d_out, 1, n, dt, s, false, true, d_ws, ws_bytes, stream);
+    Call c = make_call(d_in, d_out, 1, n, dt, s, false, d_ws, ws_bytes, stream);
+    c.level0 = true;
+    return scan_impl(c);
 }
 
 tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t dt, int s, int exclusive, void *d_in,
@@ -389,19 +550,24 @@ tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t 
     if (!h_in || !h_out || !d_in || !d_out) return TCU_ERR_INVALID_ARG;
     const size_t eb = size_t(elem_bytes(dt));
     constexpr size_t kChunk = size_t(1) << 24;                 // elements per piece (a multiple of the tile)
+    Call whole = make_call(d_in, d_out, 1, n, dt, s, exclusive != 0, d_ws, ws_bytes, stream);
+    const tcu_status_t chk = check_call(whole);
+    if (chk != TCU_OK) return chk;
     HostPipe *pipe = (exclusive || n <= 2 * kChunk) ? nullptr : host_pipe();
     if (!pipe) {                                               // short or exclusive: one copy in, one scan, one copy out
         if (cudaMemcpyAsync(d_in, h_in, n * eb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return TCU_ERR_CUDA;
-        tcu_status_t st = scan_impl(d_in, d_out, 1, n, dt, s, exclusive != 0, false, d_ws, ws_bytes, stream);
+        tcu_status_t st = scan_impl(whole);
         if (st != TCU_OK) return st;
         if (cudaMemcpyAsync(h_out, d_out, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TCU_ERR_CUDA;
         return TCU_OK;
     }
     // Long inclusive scans are cut into pieces: the upload of piece i+1, the scan of piece i (continuing from the
-    // last output of piece i-1) and the download of piece i-1 overlap, each on its own stream.
+    // total of the pieces before it) and the download of piece i-1 overlap, each on its own stream.  The total
+    // travels as an 8-byte carry through two slots of the workspace header, used in turn.
     const uint8_t *hi = reinterpret_cast<const uint8_t *>(h_in);
     uint8_t *ho = reinterpret_cast<uint8_t *>(h_out);
     uint8_t *di = reinterpret_cast<uint8_t *>(d_in), *dout = reinterpret_cast<uint8_t *>(d_out);
+    uint64_t *slots = reinterpret_cast<WsHeader *>(d_ws)->carry_slot;      // (address arithmetic only)
     if (cudaEventRecord(pipe->start, stream) != cudaSuccess) return TCU_ERR_CUDA;    // the caller's earlier work comes first
     cudaStreamWaitEvent(pipe->up, pipe->start, 0);
     cudaStreamWaitEvent(pipe->down, pipe->start, 0);
@@ -412,8 +578,10 @@ tcu_status_t tcu_scan_host(const void *h_in, void *h_out, size_t n, tcu_dtype_t 
         if (cudaMemcpyAsync(di + lo * eb, hi + lo * eb, len * eb, cudaMemcpyHostToDevice, pipe->up) != cudaSuccess) return TCU_ERR_CUDA;
         cudaEventRecord(up_done, pipe->up);
         cudaStreamWaitEvent(stream, up_done, 0);
-        tcu_status_t st = scan_impl(di + lo * eb, dout + lo * 4, 1, len, dt, s, false, false, d_ws, ws_bytes, stream, false,
-                                    i == 0 ? nullptr : dout + (lo - 1) * 4);
+        Call c = make_call(di + lo * eb, dout + lo * 4, 1, len, dt, s, false, d_ws, ws_bytes, stream);
+        c.d_carry_in = i == 0 ? nullptr : &slots[(i - 1) & 1];
+        c.d_carry_out = &slots[i & 1];
+        tcu_status_t st = scan_impl(c);
         if (st != TCU_OK) return st;
         cudaEventRecord(scan_done, stream);
         cudaStreamWaitEvent(pipe->down, scan_done, 0);
@@ -432,11 +600,51 @@ tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream) {
     return h.error == 0 ? TCU_OK : TCU_ERR_TIMEOUT;
 }
 
-tcu_status_t tcu_scan_selftest_timeout(void *d_ws, size_t ws_bytes, unsigned limit_ms, cudaStream_t stream) {
-    if (!d_ws || ws_bytes < size_t(kHeaderBytes) + 16) return TCU_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
+tcu_status_t tcu_scan_selftest_timeout(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, size_t skip_tile,
+                                       unsigned limit_ms, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
     if (limit_ms == 0 || limit_ms > 1000) return TCU_ERR_INVALID_ARG;
-    tcu_scan_timeout_selftest_kernel<<<1, 32, 0, stream>>>(d_ws, (long long)limit_ms * 2000000LL);
+    if (n == 0 || n % kTileCols != 0 || skip_tile >= tiles_for(1, n)) return TCU_ERR_INVALID_ARG;
+    Call c = make_call(d_in, d_out, 1, n, dt, s, false, d_ws, ws_bytes, stream);
+    c.skip_tile = uint32_t(skip_tile);
+    c.spin_limit = (long long)limit_ms * 2000000LL;            // about 2 cycles per nanosecond
+    return scan_impl(c);
+}
+
+tcu_status_t tcu_reduce_total(const void *d_in, size_t n, tcu_dtype_t dt, void *d_total, void *d_ws, size_t ws_bytes,
+                              cudaStream_t stream) {
+    if (!valid_dtype(dt)) return TCU_ERR_INVALID_ARG;
+    if (!d_total || (reinterpret_cast<uintptr_t>(d_total) & 7)) return TCU_ERR_INVALID_ARG;
+    if (n > 0 && (!d_in || (reinterpret_cast<uintptr_t>(d_in) & 15))) return TCU_ERR_INVALID_ARG;
+    if (n > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
+    if (!d_ws) return TCU_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
+    if (ws_bytes < tcu_scan_workspace_bytes(1, n + kTileElems, dt, 16)) return TCU_ERR_WORKSPACE;
+    // one total per 128 x 128-element tile over the whole 16-byte pieces, then one block adds them and the
+    // few elements that are left
+    const size_t per_piece = 16 / size_t(elem_bytes(dt));
+    const uint64_t whole = uint64_t(n / per_piece) * per_piece;
+    const uint32_t tiles = uint32_t((whole + kTileElems - 1) / kTileElems);
+    if (dt == TCU_I8_I32) {
+        if (tiles) tcu_tile_totals_kernel<true><<<tiles, 256, 0, stream>>>(d_in, d_ws, whole, dt);
+        tcu_sum_totals_kernel<true><<<1, 1024, 0, stream>>>(d_ws, tiles, d_in, whole, uint32_t(n - whole), dt, d_total);
+    } else {
+        if (tiles) tcu_tile_totals_kernel<false><<<tiles, 256, 0, stream>>>(d_in, d_ws, whole, dt);
+        tcu_sum_totals_kernel<false><<<1, 1024, 0, stream>>>(d_ws, tiles, d_in, whole, uint32_t(n - whole), dt, d_total);
+    }
+    return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+}
+
+tcu_status_t tcu_carry_exclusive_prefix(const void *d_totals, size_t count, size_t index, tcu_dtype_t dt, void *d_carry,
+                                        cudaStream_t stream) {
+    if (!valid_dtype(dt)) return TCU_ERR_INVALID_ARG;
+    if (!d_carry || (reinterpret_cast<uintptr_t>(d_carry) & 7) || index > count || count > (1u << 20)) return TCU_ERR_INVALID_ARG;
+    if (count > 0 && (!d_totals || (reinterpret_cast<uintptr_t>(d_totals) & 7))) return TCU_ERR_INVALID_ARG;
+    if (dt == TCU_I8_I32)
+        tcu_carry_prefix_kernel<true><<<1, 32, 0, stream>>>(reinterpret_cast<const uint64_t *>(d_totals), uint32_t(index),
+                                                          reinterpret_cast<uint64_t *>(d_carry));
+    else
+        tcu_carry_prefix_kernel<false><<<1, 32, 0, stream>>>(reinterpret_cast<const uint64_t *>(d_totals), uint32_t(index),
+                                                           reinterpret_cast<uint64_t *>(d_carry));
     return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
 }
 
@@ -459,13 +667,15 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
     int8_t *flags = reinterpret_cast<int8_t *>(d_tmp);
     int32_t *f = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(d_tmp) + a);
     uint32_t *other = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_tmp) + a + b);
+    const tcu_status_t chk = check_call(make_call(flags, f, 1, n, TCU_I8_I32, 16, true, d_ws, ws_bytes, stream));
+    if (chk != TCU_OK) return chk;
     // 32 passes ping-pong between `other` and d_keys_out so that the last pass lands in d_keys_out
     const uint32_t *src = d_keys_in;
     for (int bit = 0; bit < 32; ++bit) {
         uint32_t *dst = (bit & 1) ? d_keys_out : other;
         const unsigned blocks4 = unsigned((n + 4 * 256 - 1) / (4 * 256));
         split_flags_kernel<<<blocks4, 256, 0, stream>>>(src, flags, n, bit);
-        tcu_status_t st = scan_impl(flags, f, 1, n, TCU_I8_I32, 16, true, false, d_ws, ws_bytes, stream);
+        tcu_status_t st = scan_impl(make_call(flags, f, 1, n, TCU_I8_I32, 16, true, d_ws, ws_bytes, stream));
         if (st != TCU_OK) return st;
         split_scatter_kernel<<<unsigned((n + 255) / 256), 256, 0, stream>>>(src, flags, f, dst, n);
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
@@ -474,34 +684,16 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
     return TCU_OK;
 }
 
-tcu_status_t tcu_scan_set_down_sweep_path(int path) {
-    if (path != 0 && path != 1) return TCU_ERR_INVALID_ARG;
-    g_down_path.store(path);
-    return TCU_OK;
-}
-
-tcu_status_t tcu_scan_set_upper_level_path(int path) {
-    if (path != 0 && path != 1) return TCU_ERR_INVALID_ARG;
-    g_upper_path.store(path);
-    return TCU_OK;
-}
-
-tcu_status_t tcu_scan_set_max_ctas(int max_ctas) {
-    if (max_ctas < 0) return TCU_ERR_INVALID_ARG;
-    g_max_ctas.store(max_ctas);
-    return TCU_OK;
-}
-
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out) {
     if (!out) return TCU_ERR_INVALID_ARG;
-    std::lock_guard<std::mutex> lk(g_stats_mutex);
-    if (!g_have_stats) return TCU_ERR_INVALID_ARG;
-    *out = g_stats;
+    if (!t_have_stats) return TCU_ERR_INVALID_ARG;
+    *out = t_stats;
     return TCU_OK;
 }
 
 #ifdef TCU_PROFILE
-// Debug build only: point the kernels at a device buffer of 64 counters per CTA.
+// Debug build only (see the debug section of tcu_scan_kernel.cuh): point the kernels at a device buffer of
+// 64 wait counters per CTA, or of 8 time stamps per tile.
 int tcu_scan_debug_set_profile_buffer(void *d_buf) {
     unsigned long long *p = reinterpret_cast<unsigned long long *>(d_buf);
     return cudaMemcpyToSymbol(tcu::g_prof, &p, sizeof(p)) == cudaSuccess ? 0 : 4;

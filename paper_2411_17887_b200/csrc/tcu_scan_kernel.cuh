@@ -25,45 +25,14 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace tcu {
 
-// ---- compile-time knobs (the defaults are the measured best; the others exist for A/B builds)
-#ifndef TCU_STORE_GROUPS
-#define TCU_STORE_GROUPS 2      // groups of four store warps (2 or 3)
-#endif
-#ifndef TCU_PREFETCH_DIST
-#define TCU_PREFETCH_DIST 256   // tiles ahead of the claimed one that are prefetched into L2 (0 = off)
-#endif
-#ifndef TCU_ST_HINT
-#define TCU_ST_HINT 0           // output stores: 0 = plain, 1 = st.global.cs (streaming), 2 = st.global.L1::no_allocate
-#endif
-#ifndef TCU_LD_HINT
-#define TCU_LD_HINT 0           // input TMA loads: 1 = L2 evict-first hint (every tile is read once)
-#endif
-#ifndef TCU_PDL
-#define TCU_PDL 1               // programmatic dependent launch: set-up overlaps the tail of the previous kernel in the stream
-#endif
-#ifndef TCU_TMA_STORE
-#define TCU_TMA_STORE 0         // 1 = write the output with TMA stores instead of st.global
-#endif
-#ifndef TCU_SLABS
-#define TCU_SLABS 2             // staging slabs per store warp in the TMA-store build
-#endif
-#ifndef TCU_SETMAXNREG
-#define TCU_SETMAXNREG 1        // move registers from the control warps to the store warps
-#endif
-#ifndef TCU_LOOKBACK
-#define TCU_LOOKBACK 1          // windows of 32 records fetched per look-back round
-#endif
-#ifndef TCU_STATIC_TILES
-#define TCU_STATIC_TILES 0      // 1 = tile j of CTA b is b + j * gridDim.x instead of the next ticket
-#endif
-#ifndef TCU_MAX_STAGES
-#define TCU_MAX_STAGES 10       // most input stages the host will ask for
-#endif
-#ifndef TCU_PIPE_STORE
-#define TCU_PIPE_STORE 0        // 1 = fetch the next 32 TMEM columns before the current ones are stored
-#endif
+// ---- fixed design parameters (each was chosen by measurement; the alternatives that lost are not kept)
+constexpr int kStoreGroups = 2;               // groups of four store warps; group g takes the tiles with j % 2 == g
+constexpr uint32_t kPrefetchDist = 256;       // tiles ahead of the claimed one that are prefetched into L2
+constexpr int kUseInStages = 10;              // most input stages the host will ask for
 
 constexpr int kTileRows = 128;          // rows of a tile = M of the MMA = TMEM lanes
 constexpr int kTileCols = 128;          // elements per tile row
@@ -73,29 +42,28 @@ constexpr int kNumTot = 8;              // TMEM accumulators of the row totals (
 constexpr int kTotCols = 16;
 constexpr int kTotBase = kNumAcc * kTileCols;            // first TMEM column of the totals ring
 static_assert(kTotBase + kNumTot * kTotCols <= 512, "TMEM has 512 columns");
-constexpr int kStoreGroups = TCU_STORE_GROUPS;           // group g takes the tiles with j % kStoreGroups == g
 constexpr int kSlabBytes = 32 * 4 * 32;                  // output staging unit: 32 columns x 32 rows of 4 bytes, written by one warp
-constexpr int kSlabsPerWarp = TCU_TMA_STORE ? TCU_SLABS : 1;   // TMA stores read the slab asynchronously: ring of slabs
-constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabsPerWarp * kSlabBytes;   // staging slabs of the store warps
+constexpr int kOutRingBytes = kStoreGroups * 4 * kSlabBytes;   // one staging slab per store warp
 constexpr int kNumCarry = 16;           // tiles a CTA may have between "row totals known" and "stored": ring of carry entries
 constexpr int kTileRing = 32;           // ring of claimed tile numbers (must exceed the tiles a CTA has in flight)
 constexpr uint32_t kNoTile = 0xFFFFFFFFu;   // "no more tiles" marker pushed through the pipeline
 constexpr int kNumLookbackWarps = 5;
 constexpr int kNumMarkers = kNumLookbackWarps;   // markers pushed: one per look-back warp
 constexpr int kMaxInStages = 12;        // size of the barrier arrays
-constexpr int kUseInStages = TCU_MAX_STAGES;
-constexpr uint32_t kPrefetchDist = TCU_PREFETCH_DIST;
-constexpr int kLookBack = TCU_LOOKBACK;
 constexpr int kAtomBytes = 128 * kTileRows;   // one 128-byte-swizzled block of 128 rows
 constexpr int kOnesBytes = 16 * 128;          // constant operand of the row-total product: 16 rows of ones
 constexpr int kDownBytes = (kStoreGroups + 1) * kAtomBytes;   // carry-product variant: one carry operand per store group + a ones operand
-constexpr int kUpperBytes = kAtomBytes + 16 * 128;   // limb variant: strictly lower triangular ones (128 x 128 int8) + limb operand
+// upper levels as products: a strictly lower triangular all-ones operand (128 x 128: one 128-byte-swizzled block of
+// int8, two of bf16) and the operand that holds the narrow terms of the 128 row totals (16 rows: 2 KB per block)
+constexpr int kUpperHalfBytes = 16 * 128;
+constexpr int kUpperBytesInt = kAtomBytes + kUpperHalfBytes;
+constexpr int kUpperBytesFloat = 2 * kAtomBytes + 2 * kUpperHalfBytes;
 constexpr int kEpilogueThreads = 128;
 // Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
-// 96 x 640 = 61440 registers), so 128 x (64 + 64 + 40 + kStoreGroups x kStoreRegs) must not exceed it:
+// 96 x 640 = 61440 registers), so 128 x (64 + 64 + 88 + kStoreGroups x kStoreRegs) must not exceed it:
 // an increase that cannot be granted would block.
-constexpr int kStoreRegs = (kStoreGroups == 3) ? 104 : 128;
-static_assert(128 * (64 + 64 + 40 + kStoreGroups * kStoreRegs) <= 61440, "register pool");
+constexpr int kStoreRegs = 128;
+static_assert(128 * (64 + 64 + 88 + kStoreGroups * kStoreRegs) <= 61440, "register pool");
 constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back (warp 3 is one more)
@@ -110,47 +78,70 @@ struct WsHeader {
     uint32_t done;       // CTAs of the running launch that have finished
     uint32_t error;      // tcu_status_t recorded by a bounded wait that ran out
     uint32_t ticket;     // next tile number to hand out (tiles are claimed in increasing order)
-    uint32_t pad[60];
+    uint64_t carry_slot[2];   // scratch for a caller that chains scans: totals handed from one launch to the next
+    uint32_t pad[56];
 };
 static_assert(sizeof(WsHeader) == kHeaderBytes, "header size");
 
+// ---- debug section (compiled only with -DTCU_PROFILE; the product build defines every macro to nothing) -------------
+// Per-CTA cycle counters of where each role waits (64 counters per CTA) and eight time stamps per tile.
 #ifdef TCU_PROFILE
-// Debug build only: per-CTA cycle counters of where each role waits (64 counters per CTA).
 __device__ unsigned long long *g_prof = nullptr;
 #define PROF_DECL long long prof_t = 0; unsigned long long prof_a[8] = {0, 0, 0, 0, 0, 0, 0, 0}; (void)prof_t;
 #define PROF_T0() prof_t = clock64()
 #define PROF_ADD(k) do { long long n_ = clock64(); prof_a[k] += (unsigned long long)(n_ - prof_t); prof_t = n_; } while (0)
 #define PROF_INC(k, v) prof_a[k] += (v)
 #define PROF_FLUSH(base, cnt) do { if (g_prof) for (int i_ = 0; i_ < (cnt); ++i_) g_prof[blockIdx.x * 64 + (base) + i_] = prof_a[i_]; } while (0)
-__device__ unsigned long long *g_trace = nullptr;   // 8 time stamps per tile
-__device__ __forceinline__ unsigned long long prof_now() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define TRACE(tile, k) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = prof_now(); } while (0)
-#define TRACE_V(tile, k, v) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = (v); } while (0)
-#define PROF_STAMP(k) do { if (g_prof && threadIdx.x == 0) g_prof[blockIdx.x * 64 + 48 + (k)] = prof_now(); } while (0)
+__device__ unsigned long long *g_trace = nullptr;
+#define TRACE(tile, k) do { if (g_trace) g_trace[size_t(tile) * 8 + (k)] = global_timer_ns(); } while (0)
 #else
-#define PROF_STAMP(k)
 #define TRACE(tile, k)
-#define TRACE_V(tile, k, v)
 #define PROF_DECL
 #define PROF_T0()
 #define PROF_ADD(k)
 #define PROF_INC(k, v)
 #define PROF_FLUSH(base, cnt)
 #endif
+// ---- end of the debug section ------------------------------------------------------------------------------------------
 
-constexpr long long kSpinLimitCycles = 2000000000LL;   // about one second at B200 clocks
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) : : "memory");
+    return t;
+}
+
+// Optional time stamps of one launch (ScanParams::stamps, normally NULL): kStampsPerCta values of %globaltimer
+// per CTA, taken by whichever thread passes the point first for the CTA's first tile.
+constexpr int kStampsPerCta = 16;
+enum Stamp {
+    kStampEntry = 0,        // kernel entered
+    kStampSetupDone = 1,    // barriers, TMEM and constant operands ready
+    kStampDepsDone = 2,     // the previous kernel of the stream has finished (global memory may be touched)
+    kStampClaimed = 3,      // first tile claimed, its load issued
+    kStampLanded = 4,       // first tile in shared memory
+    kStampPublished = 5,    // first tile's total published
+    kStampCarry = 6,        // first tile's cross-tile carry known
+    kStampStored = 7,       // first tile written
+    kStampLoopsDone = 8,    // thread 0 reached the tear-down barrier
+    kStampAllDone = 9,      // every warp reached it
+    kStampExit = 10,        // TMEM freed, launch counter updated
+    kStampTiles = 11        // (not a time) tiles this CTA processed
+};
+
+// segmented scan: what is noted about a 128-element row of the array that holds a segment start
+constexpr uint32_t kRowCutIn = 1;      // a segment starts at element 0 of the row: nothing carries into it
+constexpr uint32_t kRowHasStart = 2;   // a segment starts somewhere in the row: it hands on the sum from its last start
+constexpr long long kSpinLimitCycles = 2000000000LL;   // default limit of every wait: about one second at B200 clocks
 
 struct alignas(64) ScanParams {
     CUtensorMap tmap_in;      // (128, rows128, batch) view of the input, box 128 B x 128 rows
-    CUtensorMap tmap_out;     // (128, rows128, batch) view of the output, box 32 x 32 (used by the TMA-store variant)
     void *ws;
     void *out;                // output array (4-byte elements)
-    const void *carry_in;     // optional: one output-typed value added to every element of a single-array scan (or NULL)
+    const void *carry_in;     // optional (single array): 8-byte carry (a double, or a zero-extended uint32) that precedes the scan
+    void *carry_out;          // optional (single array): receives carry_in + the total of the full rows, in the same 8-byte form
+    unsigned long long *stamps;   // optional: kStampsPerCta time stamps per CTA (see enum Stamp)
     uint64_t scan_pitch;      // elements between consecutive scans (batched), unused for a single array
+    long long spin_limit;     // cycles after which a wait gives up
     uint32_t rows128;         // full 128-element rows of one scan
     uint32_t tiles_total;     // all tiles of the launch
     uint32_t tiles_per_row;   // tiles of one scan (carry chain restarts every tiles_per_row tiles)
@@ -160,7 +151,12 @@ struct alignas(64) ScanParams {
     uint32_t level0_only;     // debug: stop after the U_s product (no carries)
     uint32_t prefilled;       // two-sweep variant: the records already hold every tile's inclusive sum
     uint32_t down_tc;         // 16-bit input, s = 128 only: add the row carries with a tensor-core product (B_s-style down-sweep)
-    uint32_t upper_tc;        // int8 only: scan the 128 row totals with a second triangular product on 8-bit limbs
+    uint32_t upper_tc;        // scan the 128 row totals with a second triangular product on exact narrow terms (8-bit limbs / bf16 terms)
+    uint32_t skip_publish_tile;   // self-test of the bounded waits: the records of this tile are never published (kNoTile: none)
+    // segmented scan (single array): per 128-element row of the array, a flag byte (kRowCutIn, kRowHasStart) and,
+    // for rows with a start, the sum from the last start to the end of the row; NULL for an ordinary scan
+    const uint8_t *seg_rowflag;
+    const uint32_t *seg_rowval;
 };
 
 // shared-memory bookkeeping (lives at the 1024-aligned base of dynamic shared memory)
@@ -177,13 +173,17 @@ struct SmemCtl {
     uint64_t agg_slot[kNumCarry];    // tile total (bits of a double, or a zero-extended uint32)
     uint64_t carry_slot[kNumCarry];  // sum of all earlier tiles of the same scan
     uint32_t warp_tot[2][4];         // cross-warp hop of the 128-row scan (double buffered)
+    uint32_t warp_cut[2][4];         // ... and whether a segment starts in the warp's 32 rows
+    uint32_t seg_cut[kNumCarry][4];  // bit r: the carry from before the tile does not reach row r (a segment starts before it)
+    uint32_t agg_cut[kNumCarry];     // a segment starts inside the tile: its total is the sum since the last start
     uint32_t tile_of[kTileRing];     // tile number of the j-th tile claimed by this CTA
     uint32_t tmem_base;
     uint32_t epoch;
-    uint32_t carry_in_bits;          // value at *carry_in (0 when there is none)
+    uint64_t carry_in_bits;          // value at *carry_in (0 when there is none)
     uint64_t epoch_ready;            // thread 0 -> totals and look-back warps: epoch and carry_in_bits are written
     uint64_t up_done;                // limb product of the row totals -> totals warps
     uint64_t down_done[kStoreGroups];   // carry product -> store warps of a group
+    uint64_t mma_drained[2];         // after a give-up: the MMAs an issuer warp still had in flight have completed
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 2048;
@@ -191,6 +191,7 @@ static_assert(sizeof(SmemCtl) <= kCtlBytes, "control block too large");
 constexpr int kRowPrefBytes = kNumCarry * kTileRows * 4;
 constexpr int kConstOffset = kCtlBytes + kRowPrefBytes;   // 10240: 1024-aligned
 static_assert(kConstOffset % 1024 == 0, "operand regions must be 1024-byte aligned");
+
 
 // ------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -223,15 +224,6 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
-#if TCU_LD_HINT
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
-        : "memory");
-    return;
-#endif
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
@@ -243,17 +235,6 @@ __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int x
                  ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int x, int y, int z) {
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(x), "r"(y), "r"(z)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -272,15 +253,11 @@ __device__ __forceinline__ bool named_barrier_or(int id, int threads, bool pred)
 // registers, every other role few.  All four warps of a group must execute the same instruction.
 template <int N>
 __device__ __forceinline__ void reg_dec() {
-#if TCU_SETMAXNREG
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
-#endif
 }
 template <int N>
 __device__ __forceinline__ void reg_inc() {
-#if TCU_SETMAXNREG
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
-#endif
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -337,13 +314,7 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t addr, uint32_t &a, uint32_
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void st_global_v4(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-#if TCU_ST_HINT == 1
-    asm volatile("st.global.cs.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-#elif TCU_ST_HINT == 2
-    asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-#else
     asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-#endif
 }
 __device__ __forceinline__ void ld_record(const void *p, uint64_t &flag, uint64_t &val) {
     asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(flag), "=l"(val) : "l"(p) : "memory");
@@ -384,6 +355,7 @@ __device__ __forceinline__ uint32_t make_idesc(uint32_t dtype, uint32_t n) {
 struct Waiter {
     SmemCtl *ctl;
     WsHeader *hdr;
+    long long limit;
     // Wait for the phase of `bar` with the given parity; false when the wait was given up.
     __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
         if (mbar_try_wait(bar, parity)) return true;
@@ -392,7 +364,7 @@ struct Waiter {
         while (!mbar_try_wait(bar, parity)) {
             if ((++spins & 0xFF) == 0) {
                 if (ctl->abort_flag) return false;
-                if (clock64() - t0 > kSpinLimitCycles) {
+                if (clock64() - t0 > limit) {
                     ctl->abort_flag = 1;
                     atomicExch(&hdr->error, 5u);
                     return false;
@@ -451,8 +423,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *in_ring = const_region + p.b_bytes;
     uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
     uint8_t *upper_a = out_ring + kOutRingBytes;          // only present when p.upper_tc
-    uint8_t *upper_b = upper_a + kAtomBytes;
-    uint8_t *down_a = out_ring + kOutRingBytes;           // only present when p.down_tc (never together with upper_tc)
+    uint8_t *upper_b = upper_a + (IS_INT ? 1 : 2) * kAtomBytes;
+    uint8_t *down_a = upper_a + (p.upper_tc ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present when p.down_tc
     uint8_t *down_b = down_a + kStoreGroups * kAtomBytes;
 
     WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
@@ -462,19 +434,20 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     const int lane = threadIdx.x & 31;
     const uint32_t num_in = p.in_stages;
 
+    // Optional time stamps (p.stamps is NULL in normal use): each point is passed by one designated thread.
+    auto stamp = [&](int k) {
+        if (p.stamps != nullptr) p.stamps[size_t(blockIdx.x) * kStampsPerCta + k] = global_timer_ns();
+    };
+
     // ---- set-up
-    PROF_STAMP(0);
-    uint32_t first_ticket = 0;                 // (thread 0 only) first tile of this CTA
-    uint32_t prev_epoch = 0;                   // (thread 0 only) launches completed on the workspace so far
     if (threadIdx.x == 0) {
+        stamp(kStampEntry);
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&p.tmap_in)) : "memory");
-#if !TCU_PDL
-        first_ticket = TCU_STATIC_TILES ? blockIdx.x : atomicAdd(&hdr->ticket, 1u);
-        prev_epoch = ld_relaxed_u32(&hdr->epoch);
-#endif
         mbar_init(smem_u32(&ctl->epoch_ready), 1);
         mbar_init(smem_u32(&ctl->up_done), 1);
         for (int g = 0; g < kStoreGroups; ++g) mbar_init(smem_u32(&ctl->down_done[g]), 1);
+        for (int g = 0; g < 2; ++g) mbar_init(smem_u32(&ctl->mma_drained[g]), 1);
+        ctl->abort_flag = 0;
     }
     {
         // the barriers are the first kNumBarriers 64-bit words of the control block: one thread each
@@ -494,46 +467,62 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             fence_barrier_init();
         }
     }
-    if (threadIdx.x == 0) ctl->abort_flag = 0;
     if (warp == 1) {
         tmem_alloc(smem_u32(&ctl->tmem_base), 512);
         tmem_relinquish();
     }
-    // Constant operands.  Row n of the K-major storage of I (x) U_s holds column n, i.e. ones at
-    // k <= n inside the same s-block (U_s is L_s transposed: X U_s = (L_s X^T)^T).  The operand of
-    // the row-total product is all ones, so every 32-byte K-slice of it is the same block.
+    // Constant operands, written as whole 16-byte pieces (the unit of the 128-byte swizzle): piece c of row n
+    // sits at n * 128 + ((c ^ (n & 7)) << 4) inside its 128-row block.  Only the pieces the products read are
+    // written; nothing else of the region is ever looked at.
     {
-        const uint32_t one = IS_INT ? 0x01010101u : ((p.dtype == 2) ? 0x3F803F80u : 0x3C003C00u);
-        uint32_t *oz = reinterpret_cast<uint32_t *>(ones_region);
-        for (uint32_t i = threadIdx.x; i < kOnesBytes / 4; i += kThreads) oz[i] = one;
-        uint32_t *cz = reinterpret_cast<uint32_t *>(const_region);
-        for (uint32_t i = threadIdx.x; i < p.b_bytes / 4; i += kThreads) cz[i] = 0;
-        __syncthreads();
-        for (int e = threadIdx.x; e < kSeff * kSeff; e += kThreads) {
-            int n = e / kSeff, k = e % kSeff;
-            if ((n / S) == (k / S) && k <= n) {
-                int kb = k * kElemBytes;
-                int off = (kb >> 7) * kAtomBytes + n * 128 + ((((kb & 127) >> 4) ^ (n & 7)) << 4) + (kb & 15);
-                if (IS_INT) {
-                    const_region[off] = 1;
-                } else {
-                    *reinterpret_cast<uint16_t *>(const_region + off) = (p.dtype == 2) ? 0x3F80 : 0x3C00;
+        const uint32_t one16 = (p.dtype == 2) ? 0x3F80u : 0x3C00u;              // 1.0 in bf16 / fp16
+        const uint32_t ones = IS_INT ? 0x01010101u : (one16 | (one16 << 16));
+        // operand of the row-total product: all ones, so every 32-byte K-slice of it is the same block
+        if (threadIdx.x < kOnesBytes / 16) st_shared_v4(smem_u32(ones_region) + threadIdx.x * 16, ones, ones, ones, ones);
+        // I (x) U_s, K-major: row n holds column n of the matrix, i.e. ones at the k <= n of the same s-block
+        // (U_s is L_s transposed: X U_s = (L_s X^T)^T)
+        constexpr int kPerPiece = 16 / kElemBytes;                              // K entries per 16-byte piece
+        constexpr int kPiecesPerRow = kSeff / kPerPiece;                        // pieces of a row that the products read
+        const uint32_t cbase = smem_u32(const_region);
+        for (int e = threadIdx.x; e < kSeff * kPiecesPerRow; e += kThreads) {
+            const int n = e / kPiecesPerRow, c = e % kPiecesPerRow;             // (powers of two: shifts and masks)
+            const int lo = n & ~(S - 1);                                        // first k of the block that row n belongs to
+            uint32_t wd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int i = 0; i < kPerPiece; ++i) {
+                const int k = c * kPerPiece + i;
+                if (k >= lo && k <= n) {
+                    if (IS_INT) wd[i >> 2] |= 1u << (8 * (i & 3));
+                    else wd[i >> 1] |= one16 << (16 * (i & 1));
                 }
             }
+            st_shared_v4(cbase + (c >> 3) * kAtomBytes + n * 128 + (((c & 7) ^ (n & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
         }
         if (!IS_INT && p.down_tc) {
             // carry operands start as zeros (only 3 of the 16 K-entries of a row are ever written); the other
             // operand is all ones in bf16
-            for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 4; e += kThreads) reinterpret_cast<uint32_t *>(down_a)[e] = 0;
-            for (int e = threadIdx.x; e < kAtomBytes / 4; e += kThreads) reinterpret_cast<uint32_t *>(down_b)[e] = 0x3F803F80u;
+            for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 16; e += kThreads) st_shared_v4(smem_u32(down_a) + e * 16, 0u, 0u, 0u, 0u);
+            for (int e = threadIdx.x; e < kAtomBytes / 16; e += kThreads)
+                st_shared_v4(smem_u32(down_b) + e * 16, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
         }
-        if (IS_INT && p.upper_tc) {
+        if (p.upper_tc) {
             // A[m][k] = 1 for k < m: its product with a column of row totals is their exclusive scan over the rows
-            for (int e = threadIdx.x; e < kTileRows * kTileRows; e += kThreads) {
-                const int m = e >> 7, k = e & 127;
-                upper_a[m * 128 + ((((k >> 4) ^ (m & 7))) << 4) + (k & 15)] = (k < m) ? 1 : 0;
+            // (int8 ones for integer scans, bf16 ones otherwise: 16 or 8 K entries per 16-byte piece)
+            constexpr int kUpPerPiece = IS_INT ? 16 : 8;
+            constexpr int kUpPieces = kTileRows / kUpPerPiece;
+            for (int e = threadIdx.x; e < kTileRows * kUpPieces; e += kThreads) {
+                const int m = e / kUpPieces, c = e % kUpPieces;
+                uint32_t wd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                for (int i = 0; i < kUpPerPiece; ++i) {
+                    if (c * kUpPerPiece + i < m) {
+                        if (IS_INT) wd[i >> 2] |= 1u << (8 * (i & 3));
+                        else wd[i >> 1] |= 0x3F80u << (16 * (i & 1));
+                    }
+                }
+                st_shared_v4(smem_u32(upper_a) + (c >> 3) * kAtomBytes + m * 128 + (((c & 7) ^ (m & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
             }
-            for (int e = threadIdx.x; e < 16 * 128 / 4; e += kThreads) reinterpret_cast<uint32_t *>(upper_b)[e] = 0;
+            for (int e = threadIdx.x; e < (IS_INT ? 1 : 2) * kUpperHalfBytes / 16; e += kThreads) st_shared_v4(smem_u32(upper_b) + e * 16, 0u, 0u, 0u, 0u);
         }
         fence_proxy_async_smem();
     }
@@ -541,44 +530,104 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
 
-    PROF_STAMP(1);
+    if (threadIdx.x == 0) stamp(kStampSetupDone);
     // Everything above touched only this CTA's shared memory and TMEM, so under programmatic dependent launch it
     // may run while the previous kernel of the stream is still finishing.  From here on global memory is read.
-#if TCU_PDL
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
     const uint32_t tmem_base = ctl->tmem_base;
-    Waiter w{ctl, hdr};
+    Waiter w{ctl, hdr, p.spin_limit};
+    uint32_t first_ticket = 0;                 // (thread 0 only) first tile of this CTA
     uint32_t my_epoch = 0;                     // (thread 0 only) the epoch of this launch
     if (threadIdx.x == 0) {
-#if TCU_PDL
-        first_ticket = TCU_STATIC_TILES ? blockIdx.x : atomicAdd(&hdr->ticket, 1u);
-        prev_epoch = ld_relaxed_u32(&hdr->epoch);
-#endif
-        my_epoch = prev_epoch + 1;
+        stamp(kStampDepsDone);
+        first_ticket = atomicAdd(&hdr->ticket, 1u);
+        my_epoch = ld_relaxed_u32(&hdr->epoch) + 1;
         ctl->epoch = my_epoch;
-        // what precedes the whole scan (continuation of an earlier segment); only single-array calls pass one
-        ctl->carry_in_bits = p.carry_in ? *reinterpret_cast<const uint32_t *>(p.carry_in) : 0u;
+        // what precedes the whole scan (continuation of an earlier piece or shard); only single-array calls pass one
+        ctl->carry_in_bits = p.carry_in ? *reinterpret_cast<const uint64_t *>(p.carry_in) : 0ull;
         mbar_arrive(smem_u32(&ctl->epoch_ready));
     }
 
-    // The j-th tile handled by this CTA is number tile_of[j % kTileRing]: either blockIdx.x + j * gridDim.x
-    // (static order) or the next ticket from the workspace (tiles claimed at run time, in increasing order:
-    // whoever holds tile t knows that every tile before t is held by a CTA that is already running).  When
-    // the tiles run out the producer pushes kNumMarkers "no more tiles" markers through the pipeline, so
-    // that every role - and each of the look-back warps - sees one and stops.
-    // ------------------------------------------------------------------ cross-tile carry scan (role of warp 3 and warps 20-23)
+    // The j-th tile handled by this CTA is number tile_of[j % kTileRing].  Tiles are claimed at run time with a
+    // ticket counter in the workspace, in increasing order: whoever holds tile t knows that every tile before t
+    // is held by a CTA that is already running.  When the tiles run out the producer pushes kNumMarkers "no more
+    // tiles" markers through the pipeline, so that every role - and each of the look-back warps, which take the
+    // tiles in turns - meets one and stops.
+    // Sum of the totals of the tiles before `t`, back to the first tile t0 of the scan or to the nearest tile whose
+    // record already holds an inclusive sum.  Every lane fetches W records per round (distance k * 32 + lane behind
+    // the current position), so that a stretch of 32 * W predecessors costs one round trip to L2; the windows are
+    // then examined nearest first, and only a window that is actually needed is waited for.
+    auto walk = [&](auto width_tag, const int t, const int t0, const uint32_t epoch, bool &gave_up, uint32_t &rounds) -> CarryT {
+        constexpr int W = decltype(width_tag)::value;
+        CarryT sum = CarryT(0);
+        int pos = t - 1;
+        while (true) {
+            uint64_t flag[W], val[W];
+#pragma unroll
+            for (int k = 0; k < W; ++k) {
+                const int idx = pos - (k * 32 + lane);
+                flag[k] = 0;
+                val[k] = 0;
+                if (idx >= t0) ld_record(records + size_t(idx) * 16, flag[k], val[k]);
+            }
+            CarryT part = CarryT(0);
+            bool done = false;
+#pragma unroll
+            for (int k = 0; k < W; ++k) {
+                if (!done) {                               // warp-uniform
+                    const int idx = pos - (k * 32 + lane);
+                    const bool valid = idx >= t0;
+                    if (valid && static_cast<uint32_t>(flag[k] >> 2) != epoch) {
+                        const void *rec = records + size_t(idx) * 16;
+                        const long long c0 = clock64();
+                        uint32_t spins = 0;
+                        while (true) {
+                            __nanosleep(20);
+                            ld_record(rec, flag[k], val[k]);
+                            if (static_cast<uint32_t>(flag[k] >> 2) == epoch) break;
+                            if ((++spins & 0x3F) == 0 && (ctl->abort_flag || clock64() - c0 > p.spin_limit)) {
+                                gave_up = true;
+                                flag[k] = kStatusInclusive;   // treat as a chain end so that the walk stops
+                                val[k] = 0;
+                                break;
+                            }
+                        }
+                    }
+                    const bool incl = valid && ((flag[k] & 3) == kStatusInclusive);
+                    const unsigned m = __ballot_sync(0xffffffffu, incl);
+                    CarryT v = valid ? CO::dec(val[k]) : CarryT(0);
+                    if (m) {
+                        const int first = __ffs(m) - 1;    // nearest predecessor whose record is inclusive
+                        if (lane > first) v = CarryT(0);
+                        done = true;
+                    }
+                    part += v;
+                    if (pos - (k * 32 + 31) <= t0) done = true;   // the window reached the first tile of the scan
+                }
+            }
+            sum += warp_sum(part);
+            ++rounds;
+            if (done) break;
+            pos -= 32 * W;
+            if (pos < t0) break;
+        }
+        return sum;
+    };
+
+    // ------------------------------------------------------------------ cross-tile carry scan (role of warp 3 and warps 16-19)
+    // kNumLookbackWarps warps take the tiles in turn, so that the walks of the tiles in flight overlap.
     auto lookback_role = [&](const uint32_t lbw) {
         if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->epoch_ready), 0))) return;
         const uint32_t epoch = ctl->epoch;
-        const CarryT carry_in = IS_INT ? CarryT(ctl->carry_in_bits) : CarryT(__uint_as_float(ctl->carry_in_bits));
-        // ------------------------------------------------------------------ cross-tile carry scan
-        // kNumLookbackWarps warps take the tiles in turn, so that the look-backs of the tiles in flight overlap.
+        const CarryT carry_in = CO::dec(ctl->carry_in_bits);
         PROF_DECL
         PROF_T0();
         for (uint32_t j = lbw;; j += kNumLookbackWarps) {
             const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;
+            CarryT prefix = CarryT(0);
+            bool gave_up = false;
+            uint32_t rounds = 0;
             if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->agg_ready[ts]), ut & 1))) break;
             PROF_ADD(0);
             const uint32_t t = ctl->tile_of[j % kTileRing];
@@ -589,83 +638,47 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (lane == 0) TRACE(t, 4);
             const CarryT agg = CO::dec(ctl->agg_slot[ts]);
             const int t0 = static_cast<int>(t - t % p.tiles_per_row);   // first tile of this scan
-            CarryT prefix = (static_cast<int>(t) == t0) ? carry_in : CarryT(0);
-            if (static_cast<int>(t) != t0) {       // (the first tile's record was published by the totals warps)
-                int pos = static_cast<int>(t) - 1;
-                bool gave_up = false;
-                while (true) {
-                    // Every lane fetches kLookBack records at once (distance d = k * 32 + lane behind pos), so
-                    // that a window of 32 * kLookBack predecessors costs one round trip to L2.  The windows
-                    // are then examined nearest first, and only a window that is actually needed is waited
-                    // for: the walk stops at the nearest record that already holds an inclusive sum.
-                    uint64_t flag[kLookBack], val[kLookBack];
-#pragma unroll
-                    for (int k = 0; k < kLookBack; ++k) {
-                        int idx = pos - (k * 32 + lane);
-                        flag[k] = 0;
-                        val[k] = 0;
-                        if (idx >= t0) ld_record(records + size_t(idx) * 16, flag[k], val[k]);
-                    }
-                    CarryT part = CarryT(0);
-                    bool done = false;
-#pragma unroll
-                    for (int k = 0; k < kLookBack; ++k) {
-                        if (!done) {                               // warp-uniform
-                            const int idx = pos - (k * 32 + lane);
-                            const bool valid = idx >= t0;
-                            if (valid && static_cast<uint32_t>(flag[k] >> 2) != epoch) {
-                                const void *rec = records + size_t(idx) * 16;
-                                long long c0 = clock64();
-                                uint32_t spins = 0;
-                                while (true) {
-                                    __nanosleep(20);
-                                    ld_record(rec, flag[k], val[k]);
-                                    if (static_cast<uint32_t>(flag[k] >> 2) == epoch) break;
-                                    if ((++spins & 0x3F) == 0 && (ctl->abort_flag || clock64() - c0 > kSpinLimitCycles)) {
-                                        gave_up = true;
-                                        flag[k] = kStatusInclusive;   // treat as a chain end so that the walk stops
-                                        val[k] = 0;
-                                        break;
-                                    }
-                                }
-                            }
-                            const bool incl = valid && ((flag[k] & 3) == kStatusInclusive);
-                            const unsigned m = __ballot_sync(0xffffffffu, incl);
-                            CarryT v = valid ? CO::dec(val[k]) : CarryT(0);
-                            if (m) {
-                                int first = __ffs(m) - 1;          // nearest predecessor whose record is inclusive
-                                if (lane > first) v = CarryT(0);
-                                done = true;
-                            }
-                            part += v;
-                            if (pos - (k * 32 + 31) <= t0) done = true;   // the window reached the first tile of the scan
-                        }
-                    }
-                    prefix += warp_sum(part);
-                    PROF_INC(2, 1);
-                    if (done) break;
-                    pos -= 32 * kLookBack;
-                    if (pos < t0) break;
+            if (static_cast<int>(t) == t0) {
+                prefix = carry_in;                 // (the first tile's record was published by the totals warps)
+            } else {
+                // One window of 32 records per round: the later a record is read the more likely it already holds an
+                // inclusive sum.  (Measured: walks that start before the tile's own total is known, or that fetch
+                // several windows per round, cover much more ground; either costs a long scan a fifth of its
+                // throughput, and does not speed up the first tiles of a launch either.)
+                prefix = walk(std::integral_constant<int, 1>{}, static_cast<int>(t), t0, epoch, gave_up, rounds);
+                if (__any_sync(0xffffffffu, gave_up) && lane == 0) {
+                    ctl->abort_flag = 1;
+                    atomicExch(&hdr->error, 5u);
                 }
-                if (__any_sync(0xffffffffu, gave_up)) {
-                    if (lane == 0) {
-                        ctl->abort_flag = 1;
-                        atomicExch(&hdr->error, 5u);
-                    }
-                }
-                // publish even after a give-up so that successors do not wait for this tile
-                if (lane == 0 && !p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
+                // publish even after a give-up so that successors do not wait for this tile (a tile in which a
+                // segment starts has already published its final record)
+                if (lane == 0 && !p.prefilled && t != p.skip_publish_tile && !(p.seg_rowflag != nullptr && ctl->agg_cut[ts]))
+                    st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
             }
             if (lane == 0) {
                 TRACE(t, 5);
                 ctl->carry_slot[ts] = CO::enc(prefix);
                 mbar_arrive(smem_u32(&ctl->carry_ready[ts]));
+                if (p.carry_out != nullptr && t + 1 == p.tiles_total) *reinterpret_cast<uint64_t *>(p.carry_out) = CO::enc(prefix + agg);
+                if (j == 0) stamp(kStampCarry);
             }
             __syncwarp();
             PROF_ADD(1);
+            PROF_INC(2, rounds);
             PROF_INC(3, 1);
         }
         if (lane == 0) PROF_FLUSH(12 + 4 * (lbw % 4), 4);
+    };
+
+    // After a give-up an MMA issuer may leave its loop with products still in flight; TMEM must not be freed
+    // under them.  A commit completes when everything this thread issued before it has, so: commit to a
+    // barrier of its own and wait for it (bounded like every other wait).
+    auto mma_drain = [&](int which) {
+        if (!ctl->abort_flag) return;
+        const uint32_t bar = smem_u32(&ctl->mma_drained[which]);
+        mma_commit(bar);
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar, 0) && clock64() - t0 < p.spin_limit) {}
     };
 
     if (warp < 4) {
@@ -681,10 +694,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
                 PROF_ADD(0);
                 uint32_t t = kNoTile;
-                if (markers == 0) {
-                    if (j == 0) t = first_ticket;
-                    else t = TCU_STATIC_TILES ? (blockIdx.x + j * gridDim.x) : atomicAdd(&hdr->ticket, 1u);
-                }
+                if (markers == 0) t = (j == 0) ? first_ticket : atomicAdd(&hdr->ticket, 1u);
                 if (t >= p.tiles_total) t = kNoTile;
                 PROF_ADD(1);
                 PROF_INC(3, 1);
@@ -703,6 +713,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     tma_load_3d(smem_u32(in_ring + stage * kStageBytes + a * kAtomBytes), &p.tmap_in,
                                 a * (128 / kElemBytes), lt * kTileRows, scan_row, bar);
                 issued = j + 1;
+                if (j == 0) stamp(kStampClaimed);
                 // Tiles are claimed in increasing order by all CTAs, so tile t + kPrefetchDist will be claimed by
                 // somebody a few microseconds from now: start its trip from DRAM to L2 now.  Its later load then
                 // costs an L2 hit, which takes the DRAM latency - and its spread - out of the carry chain.
@@ -716,6 +727,20 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 PROF_ADD(2);
             }
             PROF_FLUSH(0, 4);
+            // This CTA draws no more tickets and has read the epoch: count it.  The last CTA of the launch to get
+            // here opens the next epoch and re-arms the ticket counter; nobody of this launch looks at either
+            // again (records are compared with the copy of the epoch in shared memory), and the next launch
+            // reads them only after this one has completed.  Doing it here, not at the end of the CTA, keeps
+            // the round trip of the atomic off the tail of the kernel.
+            {
+                const uint32_t arrived = atomicAdd(&hdr->done, 1u);
+                if (arrived == gridDim.x - 1) {
+                    hdr->done = 0;
+                    hdr->ticket = 0;
+                    __threadfence();
+                    hdr->epoch = my_epoch;
+                }
+            }
             if (ctl->abort_flag) {
                 // drain: loads already issued must land before the CTA may exit
                 uint32_t lo = issued > num_in ? issued - num_in : 0;
@@ -723,7 +748,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     uint32_t bar = smem_u32(&ctl->full[j % num_in]);
                     uint32_t par = (j / num_in) & 1;
                     long long t0 = clock64();
-                    while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinLimitCycles) {}
+                    while (!mbar_try_wait(bar, par) && clock64() - t0 < p.spin_limit) {}
                 }
             }
         }
@@ -740,6 +765,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
                 if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
                 PROF_ADD(0);
+                if (j == 0) stamp(kStampLanded);
                 if (ctl->tile_of[j % kTileRing] == kNoTile) {
                     mbar_arrive(smem_u32(&ctl->empty[stage]));
                     if (++markers == kNumMarkers) break;
@@ -765,6 +791,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 PROF_ADD(2);
             }
             PROF_FLUSH(4, 3);
+            mma_drain(0);
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ MMA issuer: row totals
@@ -801,6 +828,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 PROF_ADD(2);
             }
             PROF_FLUSH(8, 3);
+            mma_drain(1);
         }
     } else {
         lookback_role(0);
@@ -809,7 +837,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         reg_dec<64>();
         lookback_role(uint32_t(warp - kFirstLookbackWarp + 1));
     } else if (warp >= kFirstTotalsWarp) {
-        reg_dec<40>();
+        reg_dec<88>();
         // ------------------------------------------------------------------ totals (up-sweep above the product)
         // Takes the 128 row totals from the small accumulator, scans them across the rows, and
         // publishes the tile total - as soon as the tile has landed, so that the cross-tile look-back
@@ -819,7 +847,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
         const bool epoch_ok = w.wait(smem_u32(&ctl->epoch_ready), 0);
         const uint32_t epoch = ctl->epoch;
-        const CarryT carry_in = IS_INT ? CarryT(ctl->carry_in_bits) : CarryT(__uint_as_float(ctl->carry_in_bits));
+        const CarryT carry_in = CO::dec(ctl->carry_in_bits);
         uint32_t markers = 0;
         PROF_DECL
         PROF_T0();
@@ -839,45 +867,86 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 continue;
             }
             if (r == 0) TRACE(t, 2);
+            uint32_t seg_fl = 0, seg_rv = 0;                          // segmented scan: this row's notes
+            if (p.seg_rowflag != nullptr) {
+                const uint64_t row = uint64_t(t) * kTileRows + r;
+                if (row < p.rows128) {
+                    seg_fl = p.seg_rowflag[row];
+                    seg_rv = p.seg_rowval[row];
+                }
+            }
             tc_fence_after();
             const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
             tmem_ld_wait();
-            if (IS_INT && p.upper_tc) {
+            if (p.upper_tc) {
                 // Paper-faithful variant of this level: the scan over the 128 row totals is itself a product
-                // with a triangular all-ones matrix.  Row totals are int32, not a tensor-core input type, so
-                // each is split into two signed 8-bit limbs (total = 128 h + l, |total| <= 2^14), the limbs
-                // are scanned by one kind::i8 product, and the two results are recombined exactly.
-                const int32_t tot = int32_t(rowtot);
+                // with a triangular all-ones matrix, D[m][n] = sum over k < m of term n of total k.  Row totals
+                // are int32 / fp32, not tensor-core input types, so each is first split exactly into narrow
+                // terms, which become rows n of the second operand (K index = tile row):
+                //   int8 input:  two signed 8-bit limbs, total = 128 h + l (|total| <= 2^14), one kind::i8 product;
+                //   16-bit input: three bf16 terms, total = hi + mid + lo (8 significant bits each), one
+                //                 kind::f16 product with fp32 accumulation.
+                // The results are recombined afterwards (shift and add; three fp32 additions).
                 const uint32_t ub = smem_u32(upper_b);
-                const uint32_t off = ((r >> 4) << 4) + (r & 15);         // k = r inside a 128-byte row, before the swizzle
-                asm volatile("st.shared.u8 [%0], %1;" ::"r"(ub + 0 * 128 + ((((r >> 4) ^ 0) << 4) | (r & 15))), "r"(tot & 127) : "memory");
-                asm volatile("st.shared.u8 [%0], %1;" ::"r"(ub + 1 * 128 + ((((r >> 4) ^ 1) << 4) | (r & 15))), "r"((tot >> 7) & 0xFF) : "memory");
-                (void)off;
+                uint32_t exc_all, tile_total;
+                if (IS_INT) {
+                    const int32_t tot = int32_t(rowtot);
+                    asm volatile("st.shared.u8 [%0], %1;" ::"r"(ub + 0 * 128 + ((((r >> 4) ^ 0) << 4) | (r & 15))), "r"(tot & 127) : "memory");
+                    asm volatile("st.shared.u8 [%0], %1;" ::"r"(ub + 1 * 128 + ((((r >> 4) ^ 1) << 4) | (r & 15))), "r"((tot >> 7) & 0xFF) : "memory");
+                } else {
+                    const uint32_t hi = rowtot & 0xFFFF0000u;
+                    const float r1 = __uint_as_float(rowtot) - __uint_as_float(hi);
+                    const uint32_t mid = __float_as_uint(r1) & 0xFFFF0000u;
+                    const float r2 = r1 - __uint_as_float(mid);
+                    const uint32_t lo = __float_as_uint(r2) & 0xFFFF0000u;             // r2 has at most 8 significant bits
+                    // K entry r of row n: 256-byte rows in two 128-byte halves of 16 rows each (2 KB per half)
+                    const uint32_t half = ub + (r >> 6) * kUpperHalfBytes, piece = (r & 63) >> 3, within = (2 * r) & 15;
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(half + 0 * 128 + ((piece ^ 0) << 4) + within), "r"(hi >> 16) : "memory");
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(half + 1 * 128 + ((piece ^ 1) << 4) + within), "r"(mid >> 16) : "memory");
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(half + 2 * 128 + ((piece ^ 2) << 4) + within), "r"(lo >> 16) : "memory");
+                }
                 fence_proxy_async_smem();
                 named_barrier_sync(2, kEpilogueThreads);
                 if (r == 0) {
                     tc_fence_after();
-                    const uint32_t idesc = make_idesc(0, kTotCols);
+                    const uint32_t d_addr = tmem_base + kTotBase + tt * kTotCols;
+                    if (IS_INT) {
+                        const uint32_t idesc = make_idesc(0, kTotCols);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_issue<true>(tmem_base + kTotBase + tt * kTotCols, make_smem_desc(smem_u32(upper_a) + kk * 32),
-                                        make_smem_desc(ub + kk * 32), idesc, kk > 0 ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk)
+                            mma_issue<true>(d_addr, make_smem_desc(smem_u32(upper_a) + kk * 32), make_smem_desc(ub + kk * 32), idesc, kk > 0 ? 1u : 0u);
+                    } else {
+                        const uint32_t idesc = make_idesc(2, kTotCols);                // bf16 operands, fp32 accumulator
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            mma_issue<false>(d_addr, make_smem_desc(smem_u32(upper_a) + (kk >> 2) * kAtomBytes + (kk & 3) * 32),
+                                             make_smem_desc(ub + (kk >> 2) * kUpperHalfBytes + (kk & 3) * 32), idesc, kk > 0 ? 1u : 0u);
+                    }
                     mma_commit(smem_u32(&ctl->up_done));
                 }
                 (void)w.wait(smem_u32(&ctl->up_done), j & 1);              // (a wait that ran out is caught by the next vote)
                 tc_fence_after();
                 const uint32_t d0 = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
                 const uint32_t d1 = tmem_ld1(lane_base + kTotBase + tt * kTotCols + 1);
+                const uint32_t d2 = tmem_ld1(lane_base + kTotBase + tt * kTotCols + 2);
                 tmem_ld_wait();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&ctl->tot_empty[tt]));            // the small accumulator may be refilled
-                const uint32_t exc_all = d0 + (d1 << 7);                   // sum of the totals of rows 0 .. r-1
+                if (IS_INT) {
+                    exc_all = d0 + (d1 << 7);                              // sum of the totals of rows 0 .. r-1
+                    tile_total = exc_all + rowtot;
+                } else {
+                    const float e = (__uint_as_float(d0) + __uint_as_float(d1)) + __uint_as_float(d2);
+                    exc_all = __float_as_uint(e);
+                    tile_total = __float_as_uint(e + __uint_as_float(rowtot));
+                }
                 rowpref[ts * kTileRows + r] = exc_all;
                 if (r == kTileRows - 1) {
-                    const CarryT a = CarryT(exc_all + rowtot);
+                    const CarryT a = IS_INT ? CarryT(tile_total) : CarryT(__uint_as_float(tile_total));
                     const bool first = (t % p.tiles_per_row == 0);
                     const uint32_t status = first ? kStatusInclusive : kStatusPartial;
-                    if (!p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
+                    if (!p.prefilled && t != p.skip_publish_tile)
+                        st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
                     ctl->agg_slot[ts] = CO::enc(a);
                 }
                 mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
@@ -886,32 +955,114 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->tot_empty[tt]));                // the small accumulator may be refilled
-            uint32_t inc = rowtot;                                    // inclusive scan across the warp's 32 rows
+            if (p.seg_rowflag == nullptr) {
+                // ordinary scan: inclusive prefix sums of the row totals across the warp's 32 rows, one hop through
+                // shared memory across the four warps
+                uint32_t inc = rowtot;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t up = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc = add32<IS_INT>(inc, up);
+                }
+                uint32_t exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                if (lane == 0) exc = 0;
+                const int pb = j & 1;
+                if (lane == 31) ctl->warp_tot[pb][wq] = inc;
+                named_barrier_sync(2, kEpilogueThreads);
+                const uint32_t w0 = ctl->warp_tot[pb][0], w1 = ctl->warp_tot[pb][1], w2 = ctl->warp_tot[pb][2], w3 = ctl->warp_tot[pb][3];
+                uint32_t before = 0;                                  // rows of the earlier warps
+                if (wq >= 1) before = w0;
+                if (wq >= 2) before = add32<IS_INT>(before, w1);
+                if (wq >= 3) before = add32<IS_INT>(before, w2);
+                rowpref[ts * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
+                if (r == 0) {
+                    const uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
+                    const CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
+                    // the first tile of a scan has nothing before it: its total is already inclusive
+                    const bool first = (t % p.tiles_per_row == 0);
+                    const uint32_t status = first ? kStatusInclusive : kStatusPartial;
+                    if (!p.prefilled && t != p.skip_publish_tile)
+                        st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
+                    TRACE(t, 3);
+                    if (j == 0) stamp(kStampPublished);
+                    ctl->agg_slot[ts] = CO::enc(a);
+                }
+                // every thread arrives (release) after its own rowpref entry is written: the look-back warp,
+                // and through it the store warps, then see all 128 entries
+                mbar_arrive(smem_u32(&ctl->agg_ready[ts]));
+                PROF_ADD(1);
+                continue;
+            }
+            // Segmented scan: the scan over the 128 rows runs on pairs (value, cut): `cut` says that a segment starts
+            // in the row, in which case `value` is the sum from that start on and nothing before the row carries
+            // past it.
+            uint32_t inc = rowtot;
+            int cut = 0, cut_in = 0;
+            if (seg_fl & kRowHasStart) {
+                inc = seg_rv;
+                cut = 1;
+                cut_in = (seg_fl & kRowCutIn) ? 1 : 0;
+            }
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                uint32_t up = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc = add32<IS_INT>(inc, up);
+                const uint32_t up = __shfl_up_sync(0xffffffffu, inc, o);
+                const int upc = __shfl_up_sync(0xffffffffu, cut, o);
+                if (lane >= o) {
+                    if (!cut) inc = add32<IS_INT>(inc, up);
+                    cut |= upc;
+                }
             }
-            uint32_t exc = __shfl_up_sync(0xffffffffu, inc, 1);
-            if (lane == 0) exc = 0;
+            uint32_t exc = __shfl_up_sync(0xffffffffu, inc, 1);       // what the rows above hand on, inside the warp
+            int exc_cut = __shfl_up_sync(0xffffffffu, cut, 1);
+            if (lane == 0) {
+                exc = 0;
+                exc_cut = 0;
+            }
             const int pb = j & 1;
-            if (lane == 31) ctl->warp_tot[pb][wq] = inc;
+            if (lane == 31) {
+                ctl->warp_tot[pb][wq] = inc;
+                ctl->warp_cut[pb][wq] = uint32_t(cut);
+            }
             named_barrier_sync(2, kEpilogueThreads);
-            uint32_t w0 = ctl->warp_tot[pb][0], w1 = ctl->warp_tot[pb][1], w2 = ctl->warp_tot[pb][2], w3 = ctl->warp_tot[pb][3];
-            uint32_t before = 0;                                      // rows of the earlier warps
-            if (wq >= 1) before = w0;
-            if (wq >= 2) before = add32<IS_INT>(before, w1);
-            if (wq >= 3) before = add32<IS_INT>(before, w2);
-            rowpref[ts * kTileRows + r] = (wq == 0) ? exc : add32<IS_INT>(before, exc);
+            uint32_t run = 0;                                         // rows of the earlier warps / of all four warps
+            int run_cut = 0;
+            uint32_t before = 0;
+            int before_cut = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (k == wq) {
+                    before = run;
+                    before_cut = run_cut;
+                }
+                const uint32_t wv = ctl->warp_tot[pb][k];
+                if (ctl->warp_cut[pb][k]) {
+                    run = wv;
+                    run_cut = 1;
+                } else {
+                    run = add32<IS_INT>(run, wv);
+                }
+            }
+            uint32_t rp = exc_cut ? exc : ((wq == 0) ? exc : add32<IS_INT>(before, exc));
+            int rp_cut = exc_cut | before_cut;
+            if (cut_in) {                                             // a segment starts with the row: nothing carries in
+                rp = 0;
+                rp_cut = 1;
+            }
+            rowpref[ts * kTileRows + r] = rp;
+            const uint32_t cut_mask = __ballot_sync(0xffffffffu, rp_cut != 0);
+            if (lane == 0) ctl->seg_cut[ts][wq] = cut_mask;
             if (r == 0) {
-                uint32_t tile_tot = add32<IS_INT>(add32<IS_INT>(w0, w1), add32<IS_INT>(w2, w3));
-                CarryT a = IS_INT ? CarryT(tile_tot) : CarryT(__uint_as_float(tile_tot));
-                // the first tile of a scan has nothing before it: its total is already inclusive
+                CarryT a = IS_INT ? CarryT(run) : CarryT(__uint_as_float(run));
+                // the first tile of a scan has nothing before it, and a tile in which a segment starts hands on
+                // only what follows that start: in both cases its total is final at once
                 const bool first = (t % p.tiles_per_row == 0);
-                const uint32_t status = first ? kStatusInclusive : kStatusPartial;
-                if (!p.prefilled) st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
+                const uint32_t status = (first || run_cut) ? kStatusInclusive : kStatusPartial;
+                if (!p.prefilled && t != p.skip_publish_tile)
+                    st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc((first && !run_cut) ? a + carry_in : a));
                 TRACE(t, 3);
+                if (j == 0) stamp(kStampPublished);
                 ctl->agg_slot[ts] = CO::enc(a);
+                ctl->agg_cut[ts] = uint32_t(run_cut);
             }
             // every thread arrives (release) after its own rowpref entry is written: the look-back warp,
             // and through it the store warps, then see all 128 entries
@@ -929,23 +1080,27 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         const int wq = warp & 3;                                    // TMEM lane quarter this warp may read
         const int r = wq * 32 + lane;                               // tile row owned by this thread
         const uint32_t lane_base = tmem_base + (uint32_t(wq * 32) << 16);
-        const uint32_t slab0 = smem_u32(out_ring) + (warp - kFirstStoreWarp) * kSlabsPerWarp * kSlabBytes;
-        uint32_t slab_counter = 0;
-        (void)slab_counter;
+        const uint32_t slab0 = smem_u32(out_ring) + (warp - kFirstStoreWarp) * kSlabBytes;
         const int sub = lane >> 3, piece = lane & 7;                // read-back role: row sub (+4i) of the slab, 16-byte piece
         uint32_t *const out32 = reinterpret_cast<uint32_t *>(p.out);
+        // The carry-product variant makes the four warps of a group meet at a barrier inside the loop, so
+        // there they must also leave the loop together: the outcome of every wait is then voted on by the
+        // whole group.  In the default path a warp shares no barrier with the others and votes alone.
+        const bool carry_product = !IS_INT && S == 128 && p.down_tc && !p.level0_only;
+        auto gave_up = [&](bool ok) {
+            return carry_product ? named_barrier_or(3 + group, kEpilogueThreads, !ok) : !__all_sync(0xffffffffu, ok);
+        };
         PROF_DECL
         PROF_T0();
+        uint32_t stored = 0;
         for (uint32_t j = group;; j += kStoreGroups) {
             const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;
             const uint32_t slot = j % kNumAcc, ua = j / kNumAcc;
-            bool ok = w.wait(smem_u32(&ctl->carry_ready[ts]), ut & 1);
-            if (!__all_sync(0xffffffffu, ok)) break;
+            if (gave_up(w.wait(smem_u32(&ctl->carry_ready[ts]), ut & 1))) break;
             PROF_ADD(0);
             const uint32_t t = ctl->tile_of[j % kTileRing];
-            if (t == kNoTile) break;
-            ok = w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1);
-            if (!__all_sync(0xffffffffu, ok)) break;
+            if (t == kNoTile) break;                                  // (the same for the whole group)
+            if (gave_up(w.wait(smem_u32(&ctl->acc_full[slot]), ua & 1))) break;
             PROF_ADD(1);
             PROF_INC(5, 1);
             if (lane == 0 && wq == 0) TRACE(t, 6);
@@ -954,6 +1109,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             uint32_t base;                                            // sum of everything before this row
             {
                 CarryT carry = CO::dec(ctl->carry_slot[ts]);
+                // segmented scan: a segment starts before this row, inside the tile
+                if (p.seg_rowflag != nullptr && ((ctl->seg_cut[ts][wq] >> lane) & 1u)) carry = CarryT(0);
                 uint32_t rp = rowpref[ts * kTileRows + r];
                 if (IS_INT) base = uint32_t(carry) + rp;
                 else base = __float_as_uint(static_cast<float>(double(carry) + double(__uint_as_float(rp))));
@@ -962,7 +1119,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (level0) base = 0;
             uint32_t run = base;                                      // sum of everything before the current chunk
             uint32_t prev = base;                                     // value of the element to the left (exclusive form)
-            if (!IS_INT && S == 128 && p.down_tc && !level0) {
+            if (carry_product) {
                 // Paper-faithful variant of the down-sweep (the B_s product: one carry added to a whole vector):
                 // the accumulator gets D += C * 1, where row r of C holds the row's carry split exactly into
                 // three bf16 terms and 1 is an all-ones operand.  128 x 128 x 16 multiply-adds for 16 Ki useful
@@ -984,7 +1141,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                                      make_idesc(2, kTileCols), 1u);
                     mma_commit(smem_u32(&ctl->down_done[group]));
                 }
-                if (!__all_sync(0xffffffffu, w.wait(smem_u32(&ctl->down_done[group]), (j / kStoreGroups) & 1))) break;
+                if (gave_up(w.wait(smem_u32(&ctl->down_done[group]), (j / kStoreGroups) & 1))) break;
                 tc_fence_after();
                 run = 0;                                              // the carry is inside the accumulator now
             }
@@ -1010,25 +1167,6 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 #pragma unroll
                     for (int c = 0; c < 32; ++c) o[c] = d[c];
                 }
-                // fetch the next 32 columns while this chunk is transposed and stored
-                if (TCU_PIPE_STORE && q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
-#if TCU_TMA_STORE
-                if (lane == 0) bulk_wait_read<kSlabsPerWarp - 1>();    // the slab about to be written has been drained
-                __syncwarp();
-                const uint32_t slab = slab0 + (slab_counter % kSlabsPerWarp) * kSlabBytes;
-                const uint32_t buf = slab + lane * 128;
-#pragma unroll
-                for (int c4 = 0; c4 < 8; ++c4)
-                    st_shared_v4(buf + ((c4 ^ (lane & 7)) << 4), o[4 * c4], o[4 * c4 + 1], o[4 * c4 + 2], o[4 * c4 + 3]);
-                fence_proxy_async_smem();
-                __syncwarp();
-                PROF_ADD(3);
-                if (lane == 0) {
-                    tma_store_3d(&p.tmap_out, slab, q * 32, row0, scan_row);
-                    bulk_commit();
-                }
-                ++slab_counter;
-#else
                 const uint32_t slab = slab0;
                 __syncwarp();                                         // the slab has been read back by every lane
                 const uint32_t buf = slab + lane * 128;
@@ -1049,38 +1187,31 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     if (rr < rows_here)
                         st_global_v4(gbase + size_t(rr) * kTileCols + q * 32, a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
                 }
-#endif
                 PROF_ADD(4);
-                if (!TCU_PIPE_STORE && q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
+                if (q < 3) tmem_ld32(lane_base + slot * kTileCols + (q + 1) * 32, d);
             }
-            if (lane == 0 && wq == 0) TRACE(t, 7);
+            if (lane == 0 && wq == 0) {
+                TRACE(t, 7);
+                if (j == 0) stamp(kStampStored);
+            }
+            ++stored;
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->acc_empty[slot]));
             // the carry ring entry of this tile (row prefixes, carry, barriers) may be reused
             mbar_arrive(smem_u32(&ctl->ring_free[ts]));
         }
-        if (TCU_TMA_STORE && lane == 0) bulk_wait_all();
         if (lane == 0 && wq == 0) PROF_FLUSH(32 + 8 * group, 6);
+        if (lane == 0 && wq == 0 && p.stamps != nullptr) p.stamps[size_t(blockIdx.x) * kStampsPerCta + kStampTiles + group] = stored;
     }
 
     // ---- tear-down
-    PROF_STAMP(2);
+    if (threadIdx.x == 0) stamp(kStampLoopsDone);
     tc_fence_before();
     __syncthreads();
-    PROF_STAMP(3);
+    if (threadIdx.x == 0) stamp(kStampAllDone);
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
-    if (threadIdx.x == 0) {
-        __threadfence();
-        uint32_t old = atomicAdd(&hdr->done, 1u);
-        if (old == gridDim.x - 1) {          // last CTA: the launch is over, open the next epoch
-            hdr->done = 0;
-            hdr->ticket = 0;
-            __threadfence();
-            hdr->epoch = my_epoch;
-        }
-    }
-    PROF_STAMP(4);
+    if (threadIdx.x == 0) stamp(kStampExit);
 }
 
 // Tail of a single-array scan: the n % 128 elements after the last full 128-element row.
@@ -1088,7 +1219,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 // last tile (or nothing when there is no full row).
 template <bool IS_INT, bool EXCL>
 __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start0, size_t pitch, uint32_t count, const void *ws,
-                                     uint32_t tiles_per_row, uint32_t dtype, const void *carry_in) {
+                                     uint32_t tiles_per_row, uint32_t dtype, const void *carry_in, void *carry_out) {
     // one block per scan (blockIdx.x = row of a batched scan)
     const size_t start = start0 + size_t(blockIdx.x) * pitch;
     const uint32_t tiles = (blockIdx.x + 1) * tiles_per_row;      // index + 1 of this scan's last tile record
@@ -1098,8 +1229,7 @@ __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start0, s
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
     CarryT carry = CarryT(0);
     if (carry_in && tiles_per_row == 0) {       // no full row before the tail: the continuation value is all there is
-        const uint32_t bits = *reinterpret_cast<const uint32_t *>(carry_in);
-        carry = IS_INT ? CarryT(bits) : CarryT(__uint_as_float(bits));
+        carry = CO::dec(*reinterpret_cast<const uint64_t *>(carry_in));
     }
     if (tiles_per_row > 0) {
         uint64_t flag, val;
@@ -1134,6 +1264,8 @@ __global__ void tcu_scan_tail_kernel(const void *in, void *out, size_t start0, s
     if (tid < int(count)) {
         if (IS_INT) reinterpret_cast<uint32_t *>(out)[start + tid] = uint32_t(y);
         else reinterpret_cast<float *>(out)[start + tid] = float(y);
+        // the total of the whole array, for a caller that continues the scan elsewhere (single arrays only)
+        if (carry_out != nullptr && tid == int(count) - 1) *reinterpret_cast<uint64_t *>(carry_out) = CO::enc(before + inc);
     }
 }
 
@@ -1238,25 +1370,187 @@ __global__ void __launch_bounds__(1024) tcu_totals_scan_kernel(void *ws, uint32_
     }
 }
 
-// Self-test of the bounded wait: one warp polls a tile record that nothing publishes, with a short
-// limit, records TCU_ERR_TIMEOUT in the workspace header exactly as the scan kernel does, and returns.
-__global__ void tcu_scan_timeout_selftest_kernel(void *ws, long long limit_cycles) {
-    WsHeader *hdr = reinterpret_cast<WsHeader *>(ws);
-    const uint8_t *rec = reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes;
-    const uint32_t epoch = ld_relaxed_u32(&hdr->epoch) + 1;     // a launch that never happens
-    uint64_t flag = 0, val = 0;
-    const long long c0 = clock64();
-    bool gave_up = false;
-    while (true) {
-        __nanosleep(100);
-        ld_record(rec, flag, val);
-        if (static_cast<uint32_t>(flag >> 2) == epoch) break;
-        if (clock64() - c0 > limit_cycles) {
-            gave_up = true;
-            break;
+// ---- segmented scan (Section 2.2 with caller-given segments): the rows that hold a segment start ---------------
+// The array is cut into rows of 128 elements, counted from its start.  A row in which no segment starts belongs to
+// one segment and goes through the tensor-core path unchanged.  A row that holds starts is summarised for that path
+// by two values: whether a segment starts at its first element (then nothing carries into the row) and the sum from
+// its last start to its end (what the row hands on).  The elements of such a row from its first start on - the
+// ones the carry of the earlier rows must not reach - are scanned again here, by one warp, straight from the input.
+
+struct SegSource {
+    const uint64_t *offsets;   // num_segments + 1 values, or NULL for equal segments of `pitch` elements
+    uint64_t pitch;
+    uint64_t num_segments;
+    __device__ __forceinline__ uint64_t start(uint64_t k) const { return offsets ? offsets[k] : k * pitch; }
+};
+
+enum SegMode { kSegPrepare = 0, kSegFixup = 1, kSegTail = 2 };
+
+// One warp per segment start (modes prepare / fixup; the warp of the first start in a row does the row) or one warp
+// in all (mode tail: the incomplete row at the end of the array, which the tile kernel never stores).
+template <bool IS_INT, bool EXCL, int MODE>
+__global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, void *out, uint64_t n, SegSource seg, const void *ws,
+                                                               uint32_t tiles, uint8_t *rowflag, uint32_t *rowval, uint32_t dtype) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    using ValT = typename std::conditional<IS_INT, uint32_t, float>::type;
+    const int lane = threadIdx.x & 31;
+    const uint64_t rows128 = n / kTileCols;
+    uint64_t row, k0;                      // the row this warp handles, and the first segment start inside it
+    bool has_start = true;
+    if (MODE == kSegTail) {
+        row = rows128;
+        // first start at or after the beginning of the row (binary search; the offsets never decrease)
+        uint64_t lo = 0, hi = seg.num_segments;
+        while (lo < hi) {
+            const uint64_t mid = (lo + hi) >> 1;
+            if (seg.start(mid) < row * kTileCols) lo = mid + 1;
+            else hi = mid;
+        }
+        k0 = lo;
+        has_start = k0 < seg.num_segments && seg.start(k0) < n;
+    } else {
+        k0 = (uint64_t(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+        if (k0 >= seg.num_segments) return;
+        const uint64_t p = seg.start(k0);
+        if (p >= n) return;                                         // empty segments at the very end
+        row = p / kTileCols;
+        if (k0 > 0 && seg.start(k0 - 1) / kTileCols == row) return;     // an earlier start of the row does it
+        if (row >= rows128) return;                                 // the incomplete last row: mode tail
+    }
+    const uint64_t base = row * kTileCols;
+    const uint32_t count = uint32_t(n - base < kTileCols ? n - base : kTileCols);
+    // this lane's four elements and their start marks
+    uint32_t mark = 0;                     // bit i: a segment starts at column 4 * lane + i
+    uint32_t first_col = kTileCols, first_inner_col = kTileCols;    // first start of the row; first one that is not at column 0
+    if (has_start) {
+        for (uint64_t k = k0; k < seg.num_segments; ++k) {
+            const uint64_t p = seg.start(k);
+            if (p >= base + count) break;
+            const uint32_t c = uint32_t(p - base);
+            if ((c >> 2) == uint32_t(lane)) mark |= 1u << (c & 3);
+            if (first_col == kTileCols) first_col = c;
+            if (c > 0 && first_inner_col == kTileCols) first_inner_col = c;
         }
     }
-    if (__any_sync(0xffffffffu, gave_up) && threadIdx.x == 0) atomicExch(&hdr->error, 5u);
+    ValT x[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t c = 4 * lane + i;
+        x[i] = ValT(0);
+        if (c < count) {
+            if (IS_INT) {
+                x[i] = ValT(int32_t(reinterpret_cast<const int8_t *>(in)[base + c]));
+            } else {
+                const uint16_t b = reinterpret_cast<const uint16_t *>(in)[base + c];
+                x[i] = ValT((dtype == 2) ? __uint_as_float(uint32_t(b) << 16) : __half2float(__ushort_as_half(b)));
+            }
+        }
+    }
+    // scan with restarts: inside the lane, then across the lanes on (restarted?, value) pairs
+    ValT inc[4];
+    ValT run = ValT(0);
+    bool cut = false;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (mark & (1u << i)) {
+            run = ValT(0);
+            cut = true;
+        }
+        run += x[i];
+        inc[i] = run;
+    }
+    ValT lane_val = run;
+    bool lane_cut = cut;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const ValT v = __shfl_up_sync(0xffffffffu, lane_val, o);
+        const int f = __shfl_up_sync(0xffffffffu, int(lane_cut), o);
+        if (lane >= o) {
+            if (!lane_cut) lane_val += v;
+            lane_cut = lane_cut || (f != 0);
+        }
+    }
+    ValT before = __shfl_up_sync(0xffffffffu, lane_val, 1);              // what the lanes to the left hand on
+    int before_cut = __shfl_up_sync(0xffffffffu, int(lane_cut), 1);
+    if (lane == 0) {
+        before = ValT(0);
+        before_cut = 0;
+    }
+    if (MODE == kSegPrepare) {
+        if (lane == 31) {
+            rowflag[row] = uint8_t(kRowHasStart | (first_col == 0 ? kRowCutIn : 0));
+            rowval[row] = IS_INT ? uint32_t(lane_val) : __float_as_uint(float(lane_val));
+        }
+        return;
+    }
+    // what precedes the row in its segment (mode tail only; in mode fixup the elements before the first start
+    // were written by the tile kernel and are left alone)
+    CarryT carry = CarryT(0);
+    if (MODE == kSegTail && tiles > 0 && first_col != 0) {
+        uint64_t flag, val;
+        ld_record(reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes + size_t(tiles - 1) * 16, flag, val);
+        carry = CO::dec(val);
+    }
+    const uint32_t from = (MODE == kSegTail) ? 0u : first_inner_col;
+    bool open = !before_cut;               // still in the segment that entered the row (the carry applies)
+    ValT left = before;                    // inclusive value of the element to the left, within its segment
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t c = 4 * lane + i;
+        if (mark & (1u << i)) {
+            open = false;
+            left = ValT(0);
+        }
+        const bool restarted_in_lane = (mark & ((2u << i) - 1)) != 0;
+        const ValT incl = restarted_in_lane ? inc[i] : ValT(before + inc[i]);
+        const ValT mine = EXCL ? left : incl;
+        if ((MODE == kSegTail || c >= from) && c < count) {
+            if (IS_INT) reinterpret_cast<uint32_t *>(out)[base + c] = uint32_t(mine) + (open ? uint32_t(carry) : 0u);
+            else reinterpret_cast<float *>(out)[base + c] = open ? float(double(carry) + double(mine)) : float(mine);
+        }
+        left = incl;
+    }
+}
+
+// ---- helpers for a scan whose array is split over several devices (Section 2.2 steps 2-3 with one segment per
+// device): the total of a shard, and the exclusive prefix of the shards' totals.  Carries travel as 8-byte values
+// in the format of the tile records (a double, or a zero-extended uint32 for integer scans).
+template <bool IS_INT>
+__global__ void __launch_bounds__(1024) tcu_sum_totals_kernel(const void *ws, uint32_t tiles, const void *in, uint64_t tail_start,
+                                                              uint32_t tail_count, uint32_t dtype, void *total_out) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    __shared__ CarryT warp_part[32];
+    const uint64_t *rec = reinterpret_cast<const uint64_t *>(reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes);
+    CarryT acc = CarryT(0);
+    for (uint32_t i = threadIdx.x; i < tiles; i += blockDim.x) acc += CO::dec(rec[2 * size_t(i) + 1]);
+    if (threadIdx.x < tail_count) {           // the few elements after the last whole 16-byte piece
+        if (IS_INT) {
+            acc += CarryT(int32_t(reinterpret_cast<const int8_t *>(in)[tail_start + threadIdx.x]));
+        } else {
+            const uint16_t b = reinterpret_cast<const uint16_t *>(in)[tail_start + threadIdx.x];
+            acc += CarryT((dtype == 2) ? __uint_as_float(uint32_t(b) << 16) : __half2float(__ushort_as_half(b)));
+        }
+    }
+    acc = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        CarryT tot = CarryT(0);
+        for (int k = 0; k < int(blockDim.x >> 5); ++k) tot += warp_part[k];
+        *reinterpret_cast<uint64_t *>(total_out) = CO::enc(tot);
+    }
+}
+
+template <bool IS_INT>
+__global__ void tcu_carry_prefix_kernel(const uint64_t *totals, uint32_t index, uint64_t *carry_out) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    CarryT acc = CarryT(0);
+    for (uint32_t i = threadIdx.x; i < index; i += 32) acc += CO::dec(totals[i]);
+    acc = warp_sum(acc);
+    if (threadIdx.x == 0) *carry_out = CO::enc(acc);
 }
 
 }  // namespace tcu

@@ -26,15 +26,17 @@ def to_device(x: np.ndarray, dtype: str) -> torch.Tensor:
 class Runner:
     """Owns a workspace and calls the library; checks guard regions and device status."""
 
-    def __init__(self, max_rows: int, max_cols: int):
-        self.ws_bytes = B.tcu_scan_workspace_bytes(max_rows, max_cols, 0, 16)
+    def __init__(self, max_rows: int, max_cols: int, ws_bytes: int = None):
+        self.ws_bytes = ws_bytes if ws_bytes is not None else B.tcu_scan_workspace_bytes(max_rows, max_cols, 0, 16)
         self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device="cuda")
         self.ws_ptr = self.ws.data_ptr() + (-self.ws.data_ptr()) % 256
         B.check(B.tcu_scan_workspace_init(self.ws_ptr, self.ws_bytes, 0))
         torch.cuda.synchronize()
 
     def run(self, x: np.ndarray, dtype: str, s: int, exclusive: bool = False, level0: bool = False,
-            d_in: torch.Tensor = None) -> np.ndarray:
+            d_in: torch.Tensor = None, **options) -> np.ndarray:
+        """`options` are the keywords of binding.tcu_scan_ex (variant, upper_level_path, max_ctas, ...); the
+        call's statistics are left in self.stats."""
         rows, cols = (1, x.size) if x.ndim == 1 else x.shape
         d_in = to_device(x, dtype) if d_in is None else d_in
         n = rows * cols
@@ -45,7 +47,11 @@ class Runner:
         assert d_out.data_ptr() % 16 == 0
         stream = torch.cuda.current_stream().cuda_stream
         dt = B.DTYPES[dtype]
-        if level0:
+        self.stats = {}
+        if options:
+            rc = B.tcu_scan_ex(d_in, d_out, rows, cols, dt, s, self.ws_ptr, self.ws_bytes, stream,
+                               exclusive=int(exclusive), stats=self.stats, **options)
+        elif level0:
             rc = B.tcu_scan_level0_debug(d_in, d_out, n, dt, s, self.ws_ptr, self.ws_bytes, stream)
         elif x.ndim == 1:
             fn = B.tcu_scan_exclusive if exclusive else B.tcu_scan_inclusive
@@ -53,6 +59,8 @@ class Runner:
         else:
             rc = B.tcu_scan_batched(d_in, d_out, rows, cols, dt, s, int(exclusive), self.ws_ptr, self.ws_bytes, stream)
         B.check(rc)
+        if not options:
+            self.stats = B.tcu_scan_last_stats()
         B.check(B.tcu_scan_device_status(self.ws_ptr, stream))
         host = out.cpu().numpy()
         sent = np.int32(SENT_I) if is_int else np.float32(SENT_F)
@@ -78,8 +86,8 @@ def assert_float_close(got: np.ndarray, x: np.ndarray, dtype: str, exclusive: bo
     return float((err / tol).max())
 
 
-def check(runner: Runner, x: np.ndarray, dtype: str, s: int, exclusive: bool = False):
-    got = runner.run(x, dtype, s, exclusive)
+def check(runner: Runner, x: np.ndarray, dtype: str, s: int, exclusive: bool = False, **options):
+    got = runner.run(x, dtype, s, exclusive, **options)
     if dtype == "i8":
         assert_int_equal(got, x, exclusive)
     else:

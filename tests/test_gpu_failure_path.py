@@ -1,5 +1,7 @@
-"""The device-side waits are bounded: a wait that nothing satisfies runs out, the kernel returns,
-the host reads TCU_ERR_TIMEOUT, and the library keeps working afterwards."""
+"""The device-side waits are bounded.  The ordinary scan kernel is launched with the records of one tile
+never published and a short limit on every wait: the tiles behind it wait in vain, the kernel records the
+time-out, every role leaves its loop, copies in flight are drained, tensor memory is freed, the kernel
+returns, the host reads TCU_ERR_TIMEOUT, and the library keeps working afterwards.  Nothing faults."""
 import numpy as np
 import pytest
 import torch
@@ -8,27 +10,43 @@ from paper_2411_17887_b200 import binding as B
 from paper_2411_17887_b200 import inputs
 
 pytestmark = pytest.mark.gpu
+TILE = 128 * 128
 
 
-def test_bounded_wait_reports_timeout_and_recovers():
+@pytest.mark.parametrize("dtype,s,tiles,skip", [("i8", 16, 40, 3), ("f16", 128, 12, 0), ("i8", 64, 400, 150)])
+def test_real_kernel_wait_runs_out_and_recovers(dtype, s, tiles, skip):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from oracle import scan_oracle as so
-    n = 3 * 16384 + 5
-    ws_bytes = B.tcu_scan_workspace_bytes(1, n, 0, 16)
+    n = tiles * TILE
+    dt = B.DTYPES[dtype]
+    ws_bytes = B.tcu_scan_workspace_bytes(1, n, dt, s)
     ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
     ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
     B.check(B.tcu_scan_workspace_init(ptr, ws_bytes, 0))
     assert B.tcu_scan_device_status(ptr, 0) == B.TCU_OK
-    assert B.tcu_scan_selftest_timeout(ptr, ws_bytes, 0, 0) == B.TCU_ERR_INVALID_ARG
-    B.check(B.tcu_scan_selftest_timeout(ptr, ws_bytes, 20, 0))      # 20 ms wait on a flag nothing sets
+    x = inputs.int8_uniform(n, -127, 127, 77) if dtype == "i8" else inputs.f16_uniform(n, -1.0, 1.0, 78)
+    d_in = torch.from_numpy(x).cuda()
+    d_out = torch.empty(n, dtype=torch.int32 if dtype == "i8" else torch.float32, device="cuda")
+    # argument checks of the self-test itself
+    assert B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, skip, 0, ptr, ws_bytes, 0) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, tiles, 20, ptr, ws_bytes, 0) == B.TCU_ERR_INVALID_ARG
+    # tile `skip` never publishes; every wait gives up after 20 ms
+    B.check(B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, skip, 20, ptr, ws_bytes, 0))
     assert B.tcu_scan_device_status(ptr, 0) == B.TCU_ERR_TIMEOUT
+    # the tiles before the silent one were not affected
+    ref = so.scan(x, dtype)
+    got = d_out.cpu().numpy()
+    if dtype == "i8":
+        assert np.array_equal(got[:skip * TILE], ref["y32"][:skip * TILE])
     # the context is intact: clear the workspace and scan with it
     B.check(B.tcu_scan_workspace_init(ptr, ws_bytes, 0))
     assert B.tcu_scan_device_status(ptr, 0) == B.TCU_OK
-    x = inputs.int8_uniform(n, -127, 127, 77)
-    d_in = torch.from_numpy(x).cuda()
-    d_out = torch.empty(n, dtype=torch.int32, device="cuda")
-    B.check(B.tcu_scan_inclusive(d_in, d_out, n, B.TCU_I8_I32, 16, ptr, ws_bytes, 0))
+    d_out.fill_(0)
+    B.check(B.tcu_scan_inclusive(d_in, d_out, n, dt, s, ptr, ws_bytes, 0))
     assert B.tcu_scan_device_status(ptr, 0) == B.TCU_OK
-    assert np.array_equal(d_out.cpu().numpy(), so.scan(x, "i8")["y32"])
+    got = d_out.cpu().numpy()
+    if dtype == "i8":
+        assert np.array_equal(got, ref["y32"])
+    else:
+        assert (np.abs(got.astype(np.float64) - ref["y"]) <= so.float_tolerance(ref["a"])).all()

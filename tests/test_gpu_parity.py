@@ -95,16 +95,20 @@ def test_int_position_sensitivity(runner):
         check(runner, x, "i8", s, True)
 
 
-def test_int_wraps_modulo_2_32(runner):
-    n = 1 << 22
-    x = np.full(n, 127, np.int8)
-    x[: 1 << 21] = 127
-    big = np.concatenate([x] * 1)
-    from tests.gpu_util import check
-    got = check(runner, big, "i8", 16)
-    assert int(got[-1]) == 127 * n                       # no wrap yet at this size ...
-    xx = np.full(1 << 22, -128, np.int8)                 # ... and the most negative input value
-    check(runner, xx, "i8", 16)
+def test_int_wraps_modulo_2_32():
+    # sums that leave the int32 range: 2^26 elements of 127 reach 8.5e9 (past 2^32, wrapping twice), 2^25
+    # elements of -128 reach -4.3e9 (past -2^31); the device must hold the exact sum modulo 2^32 throughout
+    from tests.gpu_util import Runner, check
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    big = Runner(1, 1 << 26)
+    n = 1 << 26
+    got = check(big, np.full(n, 127, np.int8), "i8", 16)
+    assert int(got[-1]) == ((127 * n + 2**31) % 2**32) - 2**31 and 127 * n > 2**32
+    assert int((got[1:] < got[:-1]).sum()) == 2          # the int32 view jumps down twice: at 2^31 and at 2^31 + 2^32
+    n = 1 << 25
+    got = check(big, np.full(n, -128, np.int8), "i8", 128, True)
+    assert int(got[-1]) == ((-128 * (n - 1) + 2**31) % 2**32) - 2**31 and -128 * (n - 1) < -2**31
 
 
 @pytest.mark.parametrize("dtype", ["i8", "bf16", "f16"])
@@ -147,7 +151,7 @@ def test_two_sweep_variant_matches_oracle(runner, dtype):
         x = gen(dtype, n, 4000 + n % 911)
         d_in = to_device(x, dtype)
         out = torch.empty(n, dtype=torch.int32 if dtype == "i8" else torch.float32, device="cuda")
-        B.check(B.tcu_scan_inclusive_twosweep(d_in, out, n, B.DTYPES[dtype], s, runner.ws_ptr, runner.ws_bytes, 0))
+        B.check(B.tcu_scan_ex(d_in, out, 1, n, B.DTYPES[dtype], s, runner.ws_ptr, runner.ws_bytes, 0, variant=1))
         B.check(B.tcu_scan_device_status(runner.ws_ptr, 0))
         assert B.tcu_scan_last_stats()["variant"] == 1
         got = out.cpu().numpy()
@@ -165,35 +169,43 @@ def test_result_does_not_depend_on_the_number_of_ctas(runner):
     from paper_2411_17887_b200 import binding as B
     from tests.gpu_util import check
     x = gen("i8", 200 * TILE + 128 * 7 + 3, 99)
-    try:
-        for p in (1, 3, 32):
-            B.check(B.tcu_scan_set_max_ctas(p))
-            check(runner, x, "i8", 16)
-            assert B.tcu_scan_last_stats()["grid"] == p
-    finally:
-        B.check(B.tcu_scan_set_max_ctas(0))
-    assert B.tcu_scan_set_max_ctas(-1) == B.TCU_ERR_INVALID_ARG
+    for p in (1, 3, 32):
+        check(runner, x, "i8", 16, max_ctas=p)
+        assert runner.stats["grid"] == p
 
 
 def test_row_total_scan_on_tensor_cores_gives_the_same_integers(runner):
     # upper level as a triangular product on 8-bit limbs instead of warp shuffles (int8 input)
     from paper_2411_17887_b200 import binding as B
     from tests.gpu_util import check
-    try:
-        B.check(B.tcu_scan_set_upper_level_path(1))
-        for n, s in [(TILE, 16), (9 * TILE + 128 * 3 + 5, 64), (700 * TILE + 77, 16), (300 * TILE, 128)]:
-            x = gen("i8", n, 7000 + n % 313)
-            check(runner, x, "i8", s)
-            check(runner, x, "i8", s, True)
-            assert B.tcu_scan_last_stats()["upper_level_path"] == 1
-        extreme = np.full(5 * TILE, -128, np.int8)          # row totals of -2^14: the limb split at its limit
-        check(runner, extreme, "i8", 16)
-        check(runner, np.full(5 * TILE, 127, np.int8), "i8", 16)
-        check(runner, gen("f16", 3 * TILE, 5), "f16", 16)   # floating-point input keeps the shuffle path
-        assert B.tcu_scan_last_stats()["upper_level_path"] == 0
-    finally:
-        B.check(B.tcu_scan_set_upper_level_path(0))
-    assert B.tcu_scan_set_upper_level_path(2) == B.TCU_ERR_INVALID_ARG
+    for n, s in [(TILE, 16), (9 * TILE + 128 * 3 + 5, 64), (700 * TILE + 77, 16), (300 * TILE, 128)]:
+        x = gen("i8", n, 7000 + n % 313)
+        check(runner, x, "i8", s, upper_level_path=1)
+        check(runner, x, "i8", s, True, upper_level_path=1)
+        assert runner.stats["upper_level_path"] == 1
+    extreme = np.full(5 * TILE, -128, np.int8)          # row totals of -2^14: the limb split at its limit
+    check(runner, extreme, "i8", 16, upper_level_path=1)
+    check(runner, np.full(5 * TILE, 127, np.int8), "i8", 16, upper_level_path=1)
+    d = torch.zeros(256, dtype=torch.int8, device="cuda")
+    o = torch.zeros(256, dtype=torch.int32, device="cuda")
+    assert B.tcu_scan_ex(d, o, 1, 256, 0, 16, runner.ws_ptr, runner.ws_bytes, 0, upper_level_path=2) == B.TCU_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_row_total_scan_on_tensor_cores_floating_point(runner, dtype):
+    # the same upper level for fp32 totals: each split exactly into three bf16 terms, one triangular kind::f16
+    # product, three fp32 additions to recombine; same tolerance, and exact on input whose sums are small integers
+    from tests.gpu_util import check
+    for n, s in [(TILE, 16), (9 * TILE + 128 * 3 + 5, 64), (400 * TILE + 77, 16), (150 * TILE, 128)]:
+        x = gen(dtype, n, 7100 + n % 313)
+        check(runner, x, dtype, s, upper_level_path=1)
+        check(runner, x, dtype, s, True, upper_level_path=1)
+        assert runner.stats["upper_level_path"] == 1
+        assert runner.stats["mma_instructions"] == runner.stats["tiles"] * ((128 // max(s, 16)) * (max(s, 16) // 16) + 8 + 8)
+    got = runner.run(np.ones(1 << 22, np.float16), "f16", 16, upper_level_path=1)
+    assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
+    check(runner, gen(dtype, 7 * TILE + 3, 5), dtype, 128, upper_level_path=1, down_sweep_path=1)   # both products at once
+    assert runner.stats["upper_level_path"] == 1 and runner.stats["down_sweep_path"] == 1
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
@@ -201,20 +213,16 @@ def test_down_sweep_as_a_tensor_core_product(runner, dtype):
     # the carry of every row added by accumulator += C * ones (C = carry in three bf16 terms) instead of vector adds
     from paper_2411_17887_b200 import binding as B
     from tests.gpu_util import check
-    try:
-        B.check(B.tcu_scan_set_down_sweep_path(1))
-        for n in (TILE, 9 * TILE + 128 * 3 + 5, 400 * TILE + 77):
-            for exclusive in (False, True):
-                check(runner, gen(dtype, n, 8000 + n % 211), dtype, 128, exclusive)
-                assert B.tcu_scan_last_stats()["down_sweep_path"] == 1
-        got = runner.run(np.ones(1 << 22, np.float16), "f16", 128)          # integers up to 2^22: must stay exact
-        assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
-        check(runner, gen(dtype, 5 * TILE, 3), dtype, 16)                   # other tile sizes ignore the knob
-        assert B.tcu_scan_last_stats()["down_sweep_path"] == 0
-        check(runner, gen("i8", 5 * TILE, 4), "i8", 128)
-        assert B.tcu_scan_last_stats()["down_sweep_path"] == 0
-    finally:
-        B.check(B.tcu_scan_set_down_sweep_path(0))
+    for n in (TILE, 9 * TILE + 128 * 3 + 5, 400 * TILE + 77):
+        for exclusive in (False, True):
+            check(runner, gen(dtype, n, 8000 + n % 211), dtype, 128, exclusive, down_sweep_path=1)
+            assert runner.stats["down_sweep_path"] == 1
+    got = runner.run(np.ones(1 << 22, np.float16), "f16", 128, down_sweep_path=1)   # integers up to 2^22: must stay exact
+    assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
+    check(runner, gen(dtype, 5 * TILE, 3), dtype, 16, down_sweep_path=1)        # other tile sizes ignore the choice
+    assert runner.stats["down_sweep_path"] == 0
+    check(runner, gen("i8", 5 * TILE, 4), "i8", 128, down_sweep_path=1)
+    assert runner.stats["down_sweep_path"] == 0
 
 
 def test_many_back_to_back_launches_agree(runner):
@@ -228,16 +236,12 @@ def test_many_back_to_back_launches_agree(runner):
     ref = torch.from_numpy(so.scan(x, "i8")["y32"]).cuda()
     d_in = to_device(x, "i8")
     outs = [torch.empty(n, dtype=torch.int32, device="cuda") for _ in range(4)]
-    try:
-        for it in range(120):
-            if it % 30 == 0:
-                B.check(B.tcu_scan_set_max_ctas([0, 5, 77, 148][it // 30]))
-            out = outs[it % 4]
-            B.check(B.tcu_scan_inclusive(d_in, out, n, B.TCU_I8_I32, 16, runner.ws_ptr, runner.ws_bytes, 0))
-            if it % 4 == 3:
-                for o in outs:
-                    assert torch.equal(o, ref)
-                    o.fill_(-1)
-    finally:
-        B.check(B.tcu_scan_set_max_ctas(0))
+    for it in range(120):
+        out = outs[it % 4]
+        B.check(B.tcu_scan_ex(d_in, out, 1, n, B.TCU_I8_I32, 16, runner.ws_ptr, runner.ws_bytes, 0,
+                              max_ctas=[0, 5, 77, 148][it // 30]))
+        if it % 4 == 3:
+            for o in outs:
+                assert torch.equal(o, ref)
+                o.fill_(-1)
     B.check(B.tcu_scan_device_status(runner.ws_ptr, 0))

@@ -38,8 +38,12 @@ def test_every_declared_symbol_is_exported(B):
 
 def test_status_strings(B):
     assert B.tcu_status_string(B.TCU_OK) == "ok"
-    seen = {B.tcu_status_string(i) for i in range(6)}
-    assert len(seen) == 6 and "unknown status" not in seen
+    codes = [B.TCU_OK, B.TCU_ERR_INVALID_ARG, B.TCU_ERR_UNSUPPORTED, B.TCU_ERR_WORKSPACE, B.TCU_ERR_CUDA,
+             B.TCU_ERR_TIMEOUT, B.TCU_ERR_TOO_LARGE]
+    assert codes == list(range(7))
+    seen = {B.tcu_status_string(i) for i in codes}
+    assert len(seen) == 7 and "unknown status" not in seen      # every status of the header has its own text
+    assert B.tcu_status_string(7) == "unknown status"
     assert B.tcu_status_string(99) == "unknown status"
 
 
@@ -66,7 +70,23 @@ def test_argument_checks_return_before_any_launch(B):
     assert B.tcu_scan_exclusive(ok_in, ok_out, 10, 0, 16, None, 0) == B.TCU_ERR_WORKSPACE
     assert B.tcu_scan_exclusive(ok_in, ok_out, 1 << 20, 0, 16, ok_ws, 64) == B.TCU_ERR_WORKSPACE    # too small
     assert B.tcu_scan_inclusive(ok_in, ok_in + 64, 1 << 10, 0, 16, ok_ws, ws) == B.TCU_ERR_INVALID_ARG  # overlap
-    assert B.tcu_scan_batched(ok_in, ok_out, 4, 100, 0, 16, 0, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED  # cols % 16
+    assert B.tcu_scan_batched(ok_in, ok_out, 4, (1 << 40) + 16, 0, 16, 0, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED   # too large
+    # the general call: malformed options are refused, carries belong to single arrays only
+    assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, variant=2) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, upper_level_path=2) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_ex(ok_in, ok_out, 2, 16, 0, 16, ok_ws, ws, d_carry_in=0x9000) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_ex(ok_in, ok_out, 1, 16, 0, 16, ok_ws, ws, d_carry_in=0x9004) == B.TCU_ERR_INVALID_ARG  # 8-byte aligned
+    assert B.tcu_scan_ex(ok_in, ok_out, 1, 16, 0, 16, ok_ws, ws, variant=1, d_carry_in=0x9000) == B.TCU_ERR_UNSUPPORTED
+    assert B.tcu_scan_selftest_timeout(ok_in, ok_out, 128, 0, 16, 0, 0, ok_ws, ws) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_selftest_timeout(ok_in, ok_out, 100, 0, 16, 0, 20, ok_ws, ws) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_reduce_total(ok_in, 100, 0, None, ok_ws, ws) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_reduce_total(ok_in + 1, 100, 0, 0x9000, ok_ws, ws) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_reduce_total(ok_in, 1 << 30, 0, 0x9000, ok_ws, 64) == B.TCU_ERR_WORKSPACE
+    assert B.tcu_carry_exclusive_prefix(0x9000, 4, 5, 0, 0xA000) == B.TCU_ERR_INVALID_ARG          # index > count
+    assert B.tcu_carry_exclusive_prefix(0x9000, 4, 2, 9, 0xA000) == B.TCU_ERR_INVALID_ARG          # dtype
+    assert B.tcu_scan_inclusive_noalloc(ok_in, ok_out, (1 << 26) + 1, 0, 16) == B.TCU_ERR_TOO_LARGE
+    assert B.tcu_scan_inclusive_noalloc(ok_in, ok_out, 0, 9, 16) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_inclusive_noalloc(ok_in + 2, ok_out, 64, 0, 16) == B.TCU_ERR_INVALID_ARG
     assert B.tcu_scan_level0_debug(ok_in, ok_out, 100, 0, 16, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED
     assert B.tcu_scan_workspace_init(None, 1024, 0) == B.TCU_ERR_WORKSPACE
     assert B.tcu_scan_device_status(None, 0) == B.TCU_ERR_WORKSPACE
