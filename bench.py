@@ -296,6 +296,65 @@ def fixed_cost(args):
     print(json.dumps({"fixed_cost": report}))
 
 
+def wait_counters(args):
+    """Where each role of the kernel waits, at the headline size: loads the debug build of the library
+    (``python -m paper_2411_17887_b200.build --profile``, compiled with -DTCU_PROFILE), runs one scan per workload
+    with a counter buffer attached and prints, per role, the mean over the CTAs of the time spent in each wait.
+    Counters perturb the kernel (it runs about a quarter slower); read the proportions, not the totals."""
+    import ctypes
+    import torch
+    from paper_2411_17887_b200 import build as lib_build
+    lib = ctypes.CDLL(lib_build.build_profile())
+    vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    lib.tcu_scan_workspace_bytes.argtypes = [sz, sz, ci, ci]
+    lib.tcu_scan_workspace_bytes.restype = sz
+    lib.tcu_scan_workspace_init.argtypes = [vp, sz, vp]
+    lib.tcu_scan_inclusive.argtypes = [vp, vp, sz, ci, ci, vp, sz, vp]
+    lib.tcu_scan_batched.argtypes = [vp, vp, sz, sz, ci, ci, ci, vp, sz, vp]
+    lib.tcu_scan_debug_set_profile_buffer.argtypes = [vp]
+    torch.cuda.set_device(0)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    ghz = torch.cuda.get_device_properties(0).clock_rate / 1e6 if hasattr(torch.cuda.get_device_properties(0), "clock_rate") else 1.965
+    n = 1 << 28
+    ws_bytes = lib.tcu_scan_workspace_bytes(4096, 65536, 0, 16)
+    ws = torch.zeros(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+    ws_ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+    prof = torch.zeros(sms * 64, dtype=torch.int64, device="cuda")
+    assert lib.tcu_scan_debug_set_profile_buffer(prof.data_ptr()) == 0
+    g = torch.Generator(device="cuda").manual_seed(1)
+    xi = torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8, generator=g)
+    xf = (torch.rand(n, device="cuda", generator=g) * 2 - 1).half()
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    names = {0: "producer: wait for a free input stage", 1: "producer: ticket", 2: "producer: issue loads",
+             4: "scan MMA: wait for the tile", 5: "scan MMA: wait for a free accumulator", 6: "scan MMA: issue",
+             8: "total MMA: wait for the tile", 9: "total MMA: wait for a free small accumulator", 10: "total MMA: issue",
+             12: "look-back warp: wait for the tile's total", 13: "look-back warp: walk",
+             28: "totals warps: wait", 29: "totals warps: work",
+             32: "store group 0: wait for the carry", 33: "store group 0: wait for the accumulator",
+             34: "store group 0: TMEM load", 35: "store group 0: add + stage", 36: "store group 0: read back + store"}
+    counts = {3: "tiles per CTA", 14: "look-back rounds of one warp", 15: "tiles of one look-back warp"}
+    report = []
+    for label, fn in [("C3 int8 n=2^28", lambda: lib.tcu_scan_inclusive(xi.data_ptr(), out.data_ptr(), n, 0, 16, ws_ptr, ws_bytes, st)),
+                      ("fp16 n=2^28", lambda: lib.tcu_scan_inclusive(xf.data_ptr(), out.data_ptr(), n, 1, 16, ws_ptr, ws_bytes, st)),
+                      ("C4-shaped 4096x65536 fp16", lambda: lib.tcu_scan_batched(xf.data_ptr(), out.data_ptr(), 4096, 65536, 1, 16, 0, ws_ptr, ws_bytes, st))]:
+        for _ in range(2):
+            assert fn() == 0
+        torch.cuda.synchronize()
+        prof.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        assert fn() == 0
+        e1.record()
+        torch.cuda.synchronize()
+        p = prof.cpu().numpy().reshape(sms, 64)
+        entry = {"workload": label, "us_with_counters": round(1e3 * e0.elapsed_time(e1), 1),
+                 "mean_us_per_cta": {nm: round(float(p[:, k].mean()) / (ghz * 1e3), 1) for k, nm in names.items()},
+                 "mean_count_per_cta": {nm: round(float(p[:, k].mean()), 1) for k, nm in counts.items()}}
+        report.append(entry)
+    print(json.dumps({"wait_counters": report, "sm_ghz_assumed": ghz}))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -459,6 +518,14 @@ def run_ours(args):
                 extra["C4_4096x65536_bf16"] = frac(time_extra(B, torch, xb, 4096, 65536, 2, 16, ws_ptr, ws_bytes)[0])
                 del xb
                 extra["C1_n2p16_i8"] = time_extra(B, torch, d_in, 1, 1 << 16, 0, 16, ws_ptr, ws_bytes, reps=200)[0]
+                # a plain widening copy with the same 1 : 4 read / write mix, for what that mix reaches without a scan
+                def widen():
+                    B.check(B.tcu_widen_copy_i8_i32(d_in, d_out, n, stream))
+                for _ in range(3):
+                    widen()
+                torch.cuda.synchronize()
+                ms_w = Timer(torch).loop(widen, 10)
+                extra["widening_copy_i8_i32_n2p28"] = frac({"us": round(1e3 * ms_w, 2), "GBps": round(5 * n / (ms_w * 1e-3) / 1e9, 1)})
                 # the same scans in the two-sweep structure (reduce, scan the totals, scan with every carry known)
                 extra["C3_two_sweep"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, variant=1)[0])
                 extra["f16_n2p28_two_sweep"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, variant=1)[0])
@@ -539,6 +606,8 @@ def main():
     ap.add_argument("--n-log2", type=int, default=28, help="log2 of the array length (28 = the headline workload)")
     ap.add_argument("--profile", action="store_true",
                     help="device-resident loop only (no end-to-end leg, no oracle): the command to wrap in ncu")
+    ap.add_argument("--wait-counters", action="store_true",
+                    help="debug build of the library: where each role of the kernel waits, at the headline size")
     ap.add_argument("--fixed-cost", action="store_true",
                     help="break the time of small launches (C1, C2, C5) into phases with the kernel's time stamps")
     args = ap.parse_args()
@@ -546,6 +615,8 @@ def main():
         run_reference(args)
     elif args.fixed_cost:
         fixed_cost(args)
+    elif args.wait_counters:
+        wait_counters(args)
     else:
         run_ours(args)
 

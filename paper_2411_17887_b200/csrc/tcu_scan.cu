@@ -684,6 +684,17 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
     return TCU_OK;
 }
 
+tcu_status_t tcu_widen_copy_i8_i32(const void *d_in, void *d_out, size_t n, cudaStream_t stream) {
+    if (n == 0) return TCU_OK;
+    if (!d_in || !d_out || (n % 16) != 0) return TCU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_in) & 15) || (reinterpret_cast<uintptr_t>(d_out) & 15)) return TCU_ERR_INVALID_ARG;
+    int sms = sm_count();
+    if (sms <= 0) return TCU_ERR_CUDA;
+    tcu_widen_copy_kernel<<<unsigned(sms) * 8, 256, 0, stream>>>(reinterpret_cast<const int4 *>(d_in), reinterpret_cast<int4 *>(d_out),
+                                                                uint64_t(n / 16));
+    return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+}
+
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out) {
     if (!out) return TCU_ERR_INVALID_ARG;
     if (!t_have_stats) return TCU_ERR_INVALID_ARG;

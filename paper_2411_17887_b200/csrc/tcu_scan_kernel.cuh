@@ -1515,6 +1515,24 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
     }
 }
 
+// ---- measuring aid: a plain widening copy with the scan's traffic mix (1 byte read, 4 bytes written per element), to
+// see what that mix reaches on this memory system without any scan in the way
+__global__ void __launch_bounds__(256) tcu_widen_copy_kernel(const int4 *in, int4 *out, uint64_t pieces) {
+    for (uint64_t i = uint64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < pieces; i += uint64_t(gridDim.x) * blockDim.x) {
+        const int4 v = in[i];                     // 16 int8 values
+        const int w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int4 o;
+            o.x = int(int8_t(w[k] & 0xFF));
+            o.y = int(int8_t((w[k] >> 8) & 0xFF));
+            o.z = int(int8_t((w[k] >> 16) & 0xFF));
+            o.w = int(int8_t((w[k] >> 24) & 0xFF));
+            out[4 * i + k] = o;
+        }
+    }
+}
+
 // ---- helpers for a scan whose array is split over several devices (Section 2.2 steps 2-3 with one segment per
 // device): the total of a shard, and the exclusive prefix of the shards' totals.  Carries travel as 8-byte values
 // in the format of the tile records (a double, or a zero-extended uint32 for integer scans).

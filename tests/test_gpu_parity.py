@@ -225,6 +225,18 @@ def test_down_sweep_as_a_tensor_core_product(runner, dtype):
     assert runner.stats["down_sweep_path"] == 0
 
 
+def test_widening_copy_measuring_aid():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2411_17887_b200 import binding as B
+    x = gen("i8", 5 * TILE + 16, 77)
+    d_in = torch.from_numpy(x).cuda()
+    d_out = torch.zeros(x.size, dtype=torch.int32, device="cuda")
+    B.check(B.tcu_widen_copy_i8_i32(d_in, d_out, x.size, 0))
+    assert np.array_equal(d_out.cpu().numpy(), x.astype(np.int32))
+    assert B.tcu_widen_copy_i8_i32(d_in, d_out, 17, 0) == B.TCU_ERR_INVALID_ARG
+
+
 def test_many_back_to_back_launches_agree(runner):
     # consecutive launches overlap their set-up with the previous kernel's tail and reuse one workspace:
     # every one of them must reproduce the integers of the first, whatever the number of CTAs
