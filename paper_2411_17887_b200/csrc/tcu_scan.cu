@@ -141,8 +141,10 @@ size_t round_up(size_t v, size_t to) { return (v + to - 1) / to * to; }
 size_t record_bytes(uint64_t tiles) { return size_t(kHeaderBytes) + 16 * size_t(tiles) + 16; }
 // workspace of a segmented scan of n elements: tile records, then one flag byte and one 4-byte value per row of 128
 size_t seg_flag_offset(uint64_t n) { return round_up(record_bytes(tiles_for(1, n)), 256); }
-size_t seg_val_offset(uint64_t n) { return seg_flag_offset(n) + round_up(size_t(n / kTileCols) + 1, 256); }
-size_t seg_workspace_bytes(uint64_t n) { return seg_val_offset(n) + 4 * (size_t(n / kTileCols) + 1); }
+// (both arrays are sized for whole tiles, plus the incomplete last row: the tile kernel copies them a tile at a time)
+size_t seg_rows(uint64_t n) { return size_t(tiles_for(1, n)) * kTileRows + 1; }
+size_t seg_val_offset(uint64_t n) { return seg_flag_offset(n) + round_up(seg_rows(n), 256); }
+size_t seg_workspace_bytes(uint64_t n) { return seg_val_offset(n) + round_up(4 * seg_rows(n), 256); }
 size_t needed_workspace(const Call &c) {
     return c.segmented ? seg_workspace_bytes(uint64_t(c.rows) * c.cols) : record_bytes(tiles_for(c.rows, c.cols));
 }
@@ -203,7 +205,7 @@ tcu_status_t scan_impl(const Call &c) {
     const bool upper_tc = c.upper_path == 1 && !c.segmented && !level0;
     const bool down_tc = (dt != TCU_I8_I32) && s == 128 && !level0 && c.down_path == 1 && !c.segmented;
     const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? (dt == TCU_I8_I32 ? kUpperBytesInt : kUpperBytesFloat) : 0) +
-                         (down_tc ? kDownBytes : 0) + 1024;  // + alignment slack
+                         (down_tc ? kDownBytes : 0) + (c.segmented ? kSegRingBytes : 0) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kUseInStages) in_stages = kUseInStages;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
@@ -241,7 +243,7 @@ tcu_status_t scan_impl(const Call &c) {
         seg_flag = reinterpret_cast<uint8_t *>(d_ws) + seg_flag_offset(cols);
         seg_val = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_ws) + seg_val_offset(cols));
         if (rows128 > 0) {
-            if (cudaMemsetAsync(seg_flag, 0, size_t(rows128), stream) != cudaSuccess) return TCU_ERR_CUDA;
+            if (cudaMemsetAsync(seg_flag, 0, size_t(tiles) * kTileRows, stream) != cudaSuccess) return TCU_ERR_CUDA;
             if (dt == TCU_I8_I32)
                 tcu_segment_rows_kernel<true, false, kSegPrepare><<<seg_blocks, 256, 0, stream>>>(d_in, d_out, cols, seg, d_ws, uint32_t(tiles), seg_flag, seg_val, dt);
             else

@@ -58,6 +58,8 @@ constexpr int kDownBytes = (kStoreGroups + 1) * kAtomBytes;   // carry-product v
 constexpr int kUpperHalfBytes = 16 * 128;
 constexpr int kUpperBytesInt = kAtomBytes + kUpperHalfBytes;
 constexpr int kUpperBytesFloat = 2 * kAtomBytes + 2 * kUpperHalfBytes;
+constexpr int kSegNoteBytes = kTileRows + 4 * kTileRows;   // segmented scan: per tile, a flag byte and a 4-byte value per row
+constexpr int kSegRingBytes = kNumCarry * kSegNoteBytes;  // one entry per carry-ring entry (reused only after the tile is stored)
 constexpr int kEpilogueThreads = 128;
 // Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
 // 96 x 640 = 61440 registers), so 128 x (64 + 64 + 88 + kStoreGroups x kStoreRegs) must not exceed it:
@@ -228,6 +230,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
+}
+// Untiled bulk copy global -> shared (both addresses 16-byte aligned, size a multiple of 16), completing on an mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 // Ask the TMA unit to bring a box into L2 only (no shared-memory destination, no completion signal).
 __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap *map, int x, int y, int z) {
@@ -422,6 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *const_region = ones_region + kOnesBytes;
     uint8_t *in_ring = const_region + p.b_bytes;
     uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
+    uint8_t *seg_ring = out_ring + kOutRingBytes;         // only present for a segmented scan (never together with the two below)
     uint8_t *upper_a = out_ring + kOutRingBytes;          // only present when p.upper_tc
     uint8_t *upper_b = upper_a + (IS_INT ? 1 : 2) * kAtomBytes;
     uint8_t *down_a = upper_a + (p.upper_tc ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present when p.down_tc
@@ -708,7 +717,16 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     continue;
                 }
                 TRACE(t, 0);
-                mbar_expect_tx(bar, kStageBytes);
+                const bool seg = p.seg_rowflag != nullptr;
+                mbar_expect_tx(bar, kStageBytes + (seg ? kSegNoteBytes : 0));
+                if (seg) {
+                    // the notes about the tile's rows travel with the tile: two bulk copies that complete on the
+                    // same barrier, into the entry of the tile's carry-ring slot (free again since tile j - 16 was
+                    // stored, which this claim already implies)
+                    const uint32_t dst = smem_u32(seg_ring + (j % kNumCarry) * kSegNoteBytes);
+                    bulk_load(dst, p.seg_rowflag + size_t(t) * kTileRows, kTileRows, bar);
+                    bulk_load(dst + kTileRows, p.seg_rowval + size_t(t) * kTileRows, 4 * kTileRows, bar);
+                }
                 int scan_row = t / p.tiles_per_row, lt = t % p.tiles_per_row;
 #pragma unroll
                 for (int a = 0; a < kInAtoms; ++a)
@@ -871,11 +889,10 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             if (r == 0) TRACE(t, 2);
             uint32_t seg_fl = 0, seg_rv = 0;                          // segmented scan: this row's notes
             if (p.seg_rowflag != nullptr) {
-                const uint64_t row = uint64_t(t) * kTileRows + r;
-                if (row < p.rows128) {
-                    seg_fl = p.seg_rowflag[row];
-                    seg_rv = p.seg_rowval[row];
-                }
+                // the notes of the tile's 128 rows came in with the tile (bulk copies issued by the producer)
+                const uint8_t *notes = seg_ring + ts * kSegNoteBytes;
+                seg_fl = notes[r];
+                seg_rv = reinterpret_cast<const uint32_t *>(notes + kTileRows)[r];
             }
             tc_fence_after();
             const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
@@ -1436,16 +1453,30 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
         }
     }
     ValT x[4];
+    if (count == kTileCols) {              // a whole row: one aligned 4- or 8-byte load per lane
+        if (IS_INT) {
+            const uint32_t w4 = reinterpret_cast<const uint32_t *>(reinterpret_cast<const int8_t *>(in) + base)[lane];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t c = 4 * lane + i;
-        x[i] = ValT(0);
-        if (c < count) {
-            if (IS_INT) {
-                x[i] = ValT(int32_t(reinterpret_cast<const int8_t *>(in)[base + c]));
-            } else {
-                const uint16_t b = reinterpret_cast<const uint16_t *>(in)[base + c];
-                x[i] = ValT((dtype == 2) ? __uint_as_float(uint32_t(b) << 16) : __half2float(__ushort_as_half(b)));
+            for (int i = 0; i < 4; ++i) x[i] = ValT(int32_t(int8_t((w4 >> (8 * i)) & 0xFF)));
+        } else {
+            const uint2 w8 = reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(in) + base)[lane];
+            const uint32_t h[4] = {w8.x & 0xFFFFu, w8.x >> 16, w8.y & 0xFFFFu, w8.y >> 16};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                x[i] = ValT((dtype == 2) ? __uint_as_float(h[i] << 16) : __half2float(__ushort_as_half(uint16_t(h[i]))));
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t c = 4 * lane + i;
+            x[i] = ValT(0);
+            if (c < count) {
+                if (IS_INT) {
+                    x[i] = ValT(int32_t(reinterpret_cast<const int8_t *>(in)[base + c]));
+                } else {
+                    const uint16_t b = reinterpret_cast<const uint16_t *>(in)[base + c];
+                    x[i] = ValT((dtype == 2) ? __uint_as_float(uint32_t(b) << 16) : __half2float(__ushort_as_half(b)));
+                }
             }
         }
     }
@@ -1497,9 +1528,9 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
     const uint32_t from = (MODE == kSegTail) ? 0u : first_inner_col;
     bool open = !before_cut;               // still in the segment that entered the row (the carry applies)
     ValT left = before;                    // inclusive value of the element to the left, within its segment
+    uint32_t res[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const uint32_t c = 4 * lane + i;
         if (mark & (1u << i)) {
             open = false;
             left = ValT(0);
@@ -1507,11 +1538,21 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
         const bool restarted_in_lane = (mark & ((2u << i) - 1)) != 0;
         const ValT incl = restarted_in_lane ? inc[i] : ValT(before + inc[i]);
         const ValT mine = EXCL ? left : incl;
-        if ((MODE == kSegTail || c >= from) && c < count) {
-            if (IS_INT) reinterpret_cast<uint32_t *>(out)[base + c] = uint32_t(mine) + (open ? uint32_t(carry) : 0u);
-            else reinterpret_cast<float *>(out)[base + c] = open ? float(double(carry) + double(mine)) : float(mine);
-        }
+        uint32_t bits;
+        if (IS_INT) bits = uint32_t(mine) + (open ? uint32_t(carry) : 0u);
+        else bits = __float_as_uint(open ? float(double(carry) + double(mine)) : float(mine));
+        res[i] = bits;
         left = incl;
+    }
+    // write: one 16-byte store when all four of the lane's elements are to be written, else element by element
+    uint32_t *const o32 = reinterpret_cast<uint32_t *>(out) + base + 4 * lane;
+    const uint32_t c0 = 4 * lane;
+    if ((MODE == kSegTail || c0 >= from) && c0 + 3 < count) {
+        *reinterpret_cast<uint4 *>(o32) = make_uint4(res[0], res[1], res[2], res[3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if ((MODE == kSegTail || c0 + i >= from) && c0 + i < count) o32[i] = res[i];
     }
 }
 
