@@ -530,7 +530,10 @@ def run_ours(args):
                 extra["C3_two_sweep"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, variant=1)[0])
                 extra["f16_n2p28_two_sweep"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, variant=1)[0])
                 # upper level (scan over the 128 row totals) as a tcgen05 product on exact narrow terms
-                extra["C3_upper_level_path1"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, upper_level_path=1)[0])
+                # (path 2: the chunk level inside a row as a product as well)
+                for path in (1, 2):
+                    extra[f"C3_upper_level_path{path}"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, upper_level_path=path)[0])
+                    extra[f"f16_n2p28_upper_level_path{path}"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, upper_level_path=path)[0])
                 # fp16, s = 128: carries added by a tensor-core product (the paper's B_s step) instead of vector adds
                 for path in (0, 1):
                     extra[f"f16_n2p28_s128_down_sweep_path{path}"] = frac(
@@ -597,8 +600,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the timings of the other configurations")
     ap.add_argument("--profile-dtype", default="i8", choices=["i8", "f16"], help="input type of the --profile loop")
     ap.add_argument("--profile-s", type=int, default=16, help="tile size s of the --profile loop")
-    ap.add_argument("--upper-level-path", type=int, default=0, choices=[0, 1],
-                    help="--profile loop: 1 scans the row totals with a tensor-core product on exact narrow terms")
+    ap.add_argument("--upper-level-path", type=int, default=0, choices=[0, 1, 2],
+                    help="--profile loop: 1 scans the row totals with a tensor-core product on exact narrow terms, "
+                         "2 the chunk totals of every row as well")
     ap.add_argument("--down-sweep-path", type=int, default=0, choices=[0, 1],
                     help="--profile loop: 1 adds the row carries with a tensor-core product (fp16 input, s = 128)")
     ap.add_argument("--sweep-ctas", action="store_true",

@@ -99,8 +99,12 @@ typedef struct {
                                        a strictly lower triangular all-ones matrix with the totals split
                                        into exact narrow terms (two signed 8-bit limbs for int8 input,
                                        three bf16 terms for fp16 / bf16 input), recombined afterwards.
+                                   2 = in addition, for s < 128, the carries of the 128 / s chunks of a row are
+                                       the product of the chunk totals (split the same way) with a strictly
+                                       upper triangular ones matrix, instead of a chain of additions along
+                                       the row (for s = 128 a row is one chunk and 2 means 1).
                                    Integer results are identical, floating-point results satisfy the
-                                   same tolerance. */
+                                   same tolerance.  The level across tiles stays a look-back on CUDA cores. */
     uint32_t down_sweep_path;   /* Paper Section 2, matrix B_s, and the discussion's remark that the tensor
                                    unit is used at O(1/s) in the down-sweep.  1 = fp16 / bf16 scans with
                                    s = 128 add each row's carry to the whole row by a tcgen05 product

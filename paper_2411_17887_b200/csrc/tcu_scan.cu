@@ -62,13 +62,13 @@ struct Shape {
     uint64_t rows, cols;
 };
 
-template <bool IS_INT, int S, bool EXCL>
+template <bool IS_INT, int S, bool EXCL, bool CHUNK_TC = false>
 cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
     static std::atomic<int> configured{-1};
     int dev = 0;
     cudaGetDevice(&dev);
     if (configured.load() != dev) {
-        cudaError_t e = cudaFuncSetAttribute(tcu_scan_kernel<IS_INT, S, EXCL>,
+        cudaError_t e = cudaFuncSetAttribute(tcu_scan_kernel<IS_INT, S, EXCL, CHUNK_TC>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
         if (e != cudaSuccess) return e;
         configured.store(dev);
@@ -85,15 +85,15 @@ cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStrea
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tcu_scan_kernel<IS_INT, S, EXCL>, prm);
+    return cudaLaunchKernelEx(&cfg, tcu_scan_kernel<IS_INT, S, EXCL, CHUNK_TC>, prm);
 }
 
 template <bool IS_INT, bool EXCL>
-cudaError_t dispatch_s(int s, const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
+cudaError_t dispatch_s(int s, bool chunk_tc, const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
     switch (s) {
-        case 16: return launch_main<IS_INT, 16, EXCL>(prm, grid, smem, stream);
-        case 64: return launch_main<IS_INT, 64, EXCL>(prm, grid, smem, stream);
-        default: return launch_main<IS_INT, 128, EXCL>(prm, grid, smem, stream);
+        case 16: return chunk_tc ? launch_main<IS_INT, 16, EXCL, true>(prm, grid, smem, stream) : launch_main<IS_INT, 16, EXCL>(prm, grid, smem, stream);
+        case 64: return chunk_tc ? launch_main<IS_INT, 64, EXCL, true>(prm, grid, smem, stream) : launch_main<IS_INT, 64, EXCL>(prm, grid, smem, stream);
+        default: return launch_main<IS_INT, 128, EXCL>(prm, grid, smem, stream);   // a row is one chunk: no chunk level
     }
 }
 
@@ -176,7 +176,7 @@ tcu_status_t check_call(const Call &c) {
     }
     const uint64_t tiles = tiles_for(c.rows, c.cols);
     if (tiles >= (1ull << 31)) return TCU_ERR_UNSUPPORTED;
-    if (c.max_ctas < 0 || c.upper_path < 0 || c.upper_path > 1 || c.down_path < 0 || c.down_path > 1) return TCU_ERR_INVALID_ARG;
+    if (c.max_ctas < 0 || c.upper_path < 0 || c.upper_path > 2 || c.down_path < 0 || c.down_path > 1) return TCU_ERR_INVALID_ARG;
     return TCU_OK;
 }
 
@@ -202,10 +202,11 @@ tcu_status_t scan_impl(const Call &c) {
     const int b_atoms = (seff * eb + 127) / 128;
     const uint32_t b_bytes = b_atoms == 1 ? uint32_t(seff * 128) : uint32_t(b_atoms * kAtomBytes);
     const uint32_t stage_bytes = kTileElems * eb;
-    const bool upper_tc = c.upper_path == 1 && !c.segmented && !level0;
+    const bool upper_tc = c.upper_path >= 1 && !c.segmented && !level0;
+    const bool chunk_tc = c.upper_path == 2 && s < kTileCols && !c.segmented && !level0;
     const bool down_tc = (dt != TCU_I8_I32) && s == 128 && !level0 && c.down_path == 1 && !c.segmented;
     const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? (dt == TCU_I8_I32 ? kUpperBytesInt : kUpperBytesFloat) : 0) +
-                         (down_tc ? kDownBytes : 0) + (c.segmented ? kSegRingBytes : 0) + 1024;  // + alignment slack
+                         (down_tc ? kDownBytes : 0) + (chunk_tc ? kChunkBytes : 0) + (c.segmented ? kSegRingBytes : 0) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kUseInStages) in_stages = kUseInStages;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
@@ -219,10 +220,10 @@ tcu_status_t scan_impl(const Call &c) {
     st.dtype = dt;
     st.exclusive = exclusive;
     st.variant = two_sweep ? 1 : 0;
-    st.upper_level_path = upper_tc ? 1 : 0;
+    st.upper_level_path = upper_tc ? uint32_t(c.upper_path) : 0;
     st.down_sweep_path = down_tc ? 1 : 0;
     st.tiles = tiles;
-    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? (dt == TCU_I8_I32 ? 4 : 8) : 0) + (down_tc ? 1 : 0));  // U_s products + row-total products
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? (dt == TCU_I8_I32 ? 4 : 8) : 0) + (chunk_tc ? (dt == TCU_I8_I32 ? 1 : 2) : 0) + (down_tc ? 1 : 0));  // U_s products + row-total products
     st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
     // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
     // scan over the tiles (absent for a single tile), carry add
@@ -317,9 +318,9 @@ tcu_status_t scan_impl(const Call &c) {
         st.grid = grid.x;
         cudaError_t e;
         if (dt == TCU_I8_I32)
-            e = exclusive ? dispatch_s<true, true>(s, prm, grid, smem, stream) : dispatch_s<true, false>(s, prm, grid, smem, stream);
+            e = exclusive ? dispatch_s<true, true>(s, chunk_tc, prm, grid, smem, stream) : dispatch_s<true, false>(s, chunk_tc, prm, grid, smem, stream);
         else
-            e = exclusive ? dispatch_s<false, true>(s, prm, grid, smem, stream) : dispatch_s<false, false>(s, prm, grid, smem, stream);
+            e = exclusive ? dispatch_s<false, true>(s, chunk_tc, prm, grid, smem, stream) : dispatch_s<false, false>(s, chunk_tc, prm, grid, smem, stream);
         if (e != cudaSuccess) return TCU_ERR_CUDA;
     }
     if (c.segmented) {
@@ -499,7 +500,7 @@ tcu_status_t tcu_scan_ex(const void *d_in, void *d_out, size_t rows, size_t cols
     if (opt) {
         if (opt->struct_bytes != sizeof(tcu_scan_options_t)) return TCU_ERR_INVALID_ARG;
         if (opt->variant > 1 || opt->max_ctas > (1u << 20)) return TCU_ERR_INVALID_ARG;
-        if (opt->upper_level_path > 1 || opt->down_sweep_path > 1) return TCU_ERR_INVALID_ARG;
+        if (opt->upper_level_path > 2 || opt->down_sweep_path > 1) return TCU_ERR_INVALID_ARG;
         c.exclusive = opt->exclusive != 0;
         c.two_sweep = opt->variant == 1;
         c.upper_path = int(opt->upper_level_path);

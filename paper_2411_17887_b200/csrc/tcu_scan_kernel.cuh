@@ -60,6 +60,12 @@ constexpr int kUpperBytesInt = kAtomBytes + kUpperHalfBytes;
 constexpr int kUpperBytesFloat = 2 * kAtomBytes + 2 * kUpperHalfBytes;
 constexpr int kSegNoteBytes = kTileRows + 4 * kTileRows;   // segmented scan: per tile, a flag byte and a 4-byte value per row
 constexpr int kSegRingBytes = kNumCarry * kSegNoteBytes;  // one entry per carry-ring entry (reused only after the tile is stored)
+// chunk level as a product (kernel variant CHUNK_TC): per store group an operand with the narrow terms of the chunk totals
+// of the 128 rows (one 128-byte-swizzled block), a constant operand of at most 32 rows, and 32 TMEM columns for the result
+constexpr int kChunkConstBytes = 32 * 128;
+constexpr int kChunkBytes = kStoreGroups * kAtomBytes + kChunkConstBytes;
+constexpr int kChunkNumTot = 4;         // row-total accumulators left when the chunk products take 64 TMEM columns
+constexpr int kChunkScratch = kTotBase + kChunkNumTot * kTotCols;    // first TMEM column of the chunk products' results
 constexpr int kEpilogueThreads = 128;
 // Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
 // 96 x 640 = 61440 registers), so 128 x (64 + 64 + 88 + kStoreGroups x kStoreRegs) must not exceed it:
@@ -70,6 +76,10 @@ constexpr int kFirstStoreWarp = 4;                                   // carry ad
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back (warp 3 is one more)
 constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps - 1);
+// The register re-allocation below assumes that the kernel is compiled at 96 registers per thread, which is what
+// 640 threads per CTA give.  With more threads the compiler settles on fewer (80 at 672), and a setmaxnreg.dec to a
+// value above the current allocation is an illegal instruction: do not add warps without redoing the numbers.
+static_assert(kThreads == 640, "register re-allocation is laid out for 640 threads at 96 registers");
 
 // workspace: 256-byte header, then one 16-byte record per tile
 constexpr int kHeaderBytes = 256;
@@ -186,6 +196,7 @@ struct SmemCtl {
     uint64_t up_done;                // limb product of the row totals -> totals warps
     uint64_t down_done[kStoreGroups];   // carry product -> store warps of a group
     uint64_t mma_drained[2];         // after a give-up: the MMAs an issuer warp still had in flight have completed
+    uint64_t chunk_done[kStoreGroups];  // chunk product -> store warps of a group
     volatile uint32_t abort_flag;
 };
 constexpr int kCtlBytes = 2048;
@@ -409,8 +420,10 @@ __device__ __forceinline__ uint32_t add32(uint32_t a, uint32_t b) {
 }
 
 // ------------------------------------------------------------------------------------ kernel
-template <bool IS_INT, int S, bool EXCL>
+template <bool IS_INT, int S, bool EXCL, bool CHUNK_TC = false>
 __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_constant__ ScanParams p) {
+    static_assert(!CHUNK_TC || S < kTileCols, "a row of s = 128 is one chunk: there is no chunk level");
+    constexpr int kTotRing = CHUNK_TC ? kChunkNumTot : kNumTot;   // depth of the ring of row-total accumulators
     using CO = CarryOps<IS_INT>;
     using CarryT = typename CO::T;
     constexpr int kElemBytes = IS_INT ? 1 : 2;
@@ -435,6 +448,8 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *upper_b = upper_a + (IS_INT ? 1 : 2) * kAtomBytes;
     uint8_t *down_a = upper_a + (p.upper_tc ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present when p.down_tc
     uint8_t *down_b = down_a + kStoreGroups * kAtomBytes;
+    uint8_t *chunk_a = upper_a + (p.upper_tc ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present in the CHUNK_TC variant
+    uint8_t *chunk_b = chunk_a + kStoreGroups * kAtomBytes;
 
     WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
     uint8_t *records = reinterpret_cast<uint8_t *>(p.ws) + kHeaderBytes;
@@ -456,6 +471,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         mbar_init(smem_u32(&ctl->up_done), 1);
         for (int g = 0; g < kStoreGroups; ++g) mbar_init(smem_u32(&ctl->down_done[g]), 1);
         for (int g = 0; g < 2; ++g) mbar_init(smem_u32(&ctl->mma_drained[g]), 1);
+        for (int g = 0; g < kStoreGroups; ++g) mbar_init(smem_u32(&ctl->chunk_done[g]), 1);
         ctl->abort_flag = 0;
     }
     {
@@ -532,6 +548,29 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 st_shared_v4(smem_u32(upper_a) + (c >> 3) * kAtomBytes + m * 128 + (((c & 7) ^ (m & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
             }
             for (int e = threadIdx.x; e < (IS_INT ? 1 : 2) * kUpperHalfBytes / 16; e += kThreads) st_shared_v4(smem_u32(upper_b) + e * 16, 0u, 0u, 0u, 0u);
+        }
+        if (CHUNK_TC) {
+            // Chunk level as a product: the K index of the data operand is (chunk g', term l') = kTerms g' + l', the
+            // result column is (chunk g, term l) = kTerms g + l, and the constant operand (stored K-major: row n holds
+            // column n) has ones where l' = l and g' < g: column (g, l) of the result is the sum of term l over the
+            // chunks before g - a strictly upper triangular U_{128/s}, once per term.
+            constexpr int kTerms = IS_INT ? 2 : 3, kCPerPiece = IS_INT ? 16 : 8, kCPieces = 32 / kCPerPiece;
+            for (int e = threadIdx.x; e < 32 * kCPieces; e += kThreads) {
+                const int n = e / kCPieces, c = e % kCPieces;
+                uint32_t wd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                for (int i = 0; i < kCPerPiece; ++i) {
+                    const int k = c * kCPerPiece + i;
+                    const bool used = n < kTerms * (kTileCols / S) && k < kTerms * (kTileCols / S);
+                    if (used && (k % kTerms) == (n % kTerms) && (k / kTerms) < (n / kTerms)) {
+                        if (IS_INT) wd[i >> 2] |= 1u << (8 * (i & 3));
+                        else wd[i >> 1] |= 0x3F80u << (16 * (i & 1));
+                    }
+                }
+                st_shared_v4(smem_u32(chunk_b) + n * 128 + ((c ^ (n & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
+            }
+            // the data operands start as zeros: only the first pieces of a row are ever rewritten
+            for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 16; e += kThreads) st_shared_v4(smem_u32(chunk_a) + e * 16, 0u, 0u, 0u, 0u);
         }
         fence_proxy_async_smem();
     }
@@ -823,7 +862,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             PROF_T0();
             for (uint32_t j = 0;; ++j) {
                 uint32_t stage = j % num_in, u = j / num_in;
-                uint32_t ts = j % kNumTot, ut = j / kNumTot;
+                uint32_t ts = j % kTotRing, ut = j / kTotRing;
                 if (!w.wait(smem_u32(&ctl->full[stage]), u & 1)) break;
                 PROF_ADD(0);
                 if (!w.wait(smem_u32(&ctl->tot_empty[ts]), (ut & 1) ^ 1)) break;
@@ -872,7 +911,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         PROF_DECL
         PROF_T0();
         for (uint32_t j = 0;; ++j) {
-            const uint32_t tt = j % kNumTot, utt = j / kNumTot;      // row-total accumulator in TMEM
+            const uint32_t tt = j % kTotRing, utt = j / kTotRing;    // row-total accumulator in TMEM
             const uint32_t ts = j % kNumCarry, ut = j / kNumCarry;   // carry ring entry
             // a wait that ran out is voted on, so that all 128 threads leave together
             bool ok = w.wait(smem_u32(&ctl->tot_full[tt]), utt & 1) && epoch_ok;
@@ -1106,8 +1145,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         // there they must also leave the loop together: the outcome of every wait is then voted on by the
         // whole group.  In the default path a warp shares no barrier with the others and votes alone.
         const bool carry_product = !IS_INT && S == 128 && p.down_tc && !p.level0_only;
+        const bool group_meets = carry_product || CHUNK_TC;       // (the chunk product has the same group barrier)
         auto gave_up = [&](bool ok) {
-            return carry_product ? named_barrier_or(3 + group, kEpilogueThreads, !ok) : !__all_sync(0xffffffffu, ok);
+            return group_meets ? named_barrier_or(3 + group, kEpilogueThreads, !ok) : !__all_sync(0xffffffffu, ok);
         };
         PROF_DECL
         PROF_T0();
@@ -1164,6 +1204,70 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 tc_fence_after();
                 run = 0;                                              // the carry is inside the accumulator now
             }
+            // Paper-faithful variant of the chunk level (kernel variant CHUNK_TC): the carries of the 128 / s chunks of a
+            // row are the exclusive scan of the chunk totals, here a product of the totals with a strictly upper
+            // triangular ones matrix.  The totals (the last column of every chunk in the accumulator) are int32 /
+            // fp32, so each is split exactly into narrow terms first (two 8-bit limbs, |total| <= 2^13; three bf16
+            // terms), the terms of the group's 128 rows form the data operand, one kind::i8 product (two kind::f16
+            // products) scans them, and the results are recombined.  The register chain below is then not used.
+            uint32_t chunk_carry[CHUNK_TC ? kTileCols / S : 1];
+            if (CHUNK_TC && !level0) {
+                constexpr int kChunks = kTileCols / S, kTerms = IS_INT ? 2 : 3;
+                uint32_t tot[kChunks];
+#pragma unroll
+                for (int g = 0; g < kChunks; ++g) tot[g] = tmem_ld1(lane_base + slot * kTileCols + (g + 1) * S - 1);
+                tmem_ld_wait();
+                uint32_t wd[12] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};      // K entries kTerms g + l, packed
+#pragma unroll
+                for (int g = 0; g < kChunks; ++g) {
+                    if (IS_INT) {
+                        const int32_t v = int32_t(tot[g]);
+                        const uint32_t lo = uint32_t(v & 127), hi = uint32_t((v >> 7) & 0xFF);
+                        wd[(2 * g) >> 2] |= lo << (8 * ((2 * g) & 3));
+                        wd[(2 * g + 1) >> 2] |= hi << (8 * ((2 * g + 1) & 3));
+                    } else {
+                        const uint32_t hi = tot[g] & 0xFFFF0000u;
+                        const float r1 = __uint_as_float(tot[g]) - __uint_as_float(hi);
+                        const uint32_t mid = __float_as_uint(r1) & 0xFFFF0000u;
+                        const float r2 = r1 - __uint_as_float(mid);
+                        const uint32_t lo = __float_as_uint(r2) & 0xFFFF0000u;
+                        const uint32_t term[3] = {hi >> 16, mid >> 16, lo >> 16};
+#pragma unroll
+                        for (int l = 0; l < 3; ++l) wd[(3 * g + l) >> 1] |= term[l] << (16 * ((3 * g + l) & 1));
+                    }
+                }
+                const uint32_t ca = smem_u32(chunk_a) + group * kAtomBytes;
+                const uint32_t rowa = ca + r * 128;
+                constexpr int kPiecesUsed = (kTerms * kChunks * (IS_INT ? 1 : 2) + 15) / 16;
+#pragma unroll
+                for (int c = 0; c < kPiecesUsed; ++c)
+                    st_shared_v4(rowa + ((c ^ (r & 7)) << 4), wd[4 * c], wd[4 * c + 1], wd[4 * c + 2], wd[4 * c + 3]);
+                fence_proxy_async_smem();
+                named_barrier_sync(3 + group, kEpilogueThreads);
+                const uint32_t d2 = tmem_base + kChunkScratch + group * 32;
+                if (wq == 0 && lane == 0) {
+                    tc_fence_after();
+                    if (IS_INT) {
+                        mma_issue<true>(d2, make_smem_desc(ca), make_smem_desc(smem_u32(chunk_b)), make_idesc(0, 16), 0u);
+                    } else {
+#pragma unroll
+                        for (int kk = 0; kk < 2; ++kk)
+                            mma_issue<false>(d2, make_smem_desc(ca + kk * 32), make_smem_desc(smem_u32(chunk_b) + kk * 32), make_idesc(2, 32), kk > 0 ? 1u : 0u);
+                    }
+                    mma_commit(smem_u32(&ctl->chunk_done[group]));
+                }
+                if (gave_up(w.wait(smem_u32(&ctl->chunk_done[group]), (j / kStoreGroups) & 1))) break;
+                tc_fence_after();
+                uint32_t res[kTerms * kChunks];
+#pragma unroll
+                for (int n = 0; n < kTerms * kChunks; ++n) res[n] = tmem_ld1(lane_base + kChunkScratch + group * 32 + n);
+                tmem_ld_wait();
+#pragma unroll
+                for (int g = 0; g < kChunks; ++g) {
+                    if (IS_INT) chunk_carry[g] = res[2 * g] + (res[2 * g + 1] << 7);
+                    else chunk_carry[g] = __float_as_uint((__uint_as_float(res[3 * g]) + __uint_as_float(res[3 * g + 1])) + __uint_as_float(res[3 * g + 2]));
+                }
+            }
             const uint32_t row0 = lt * kTileRows + wq * 32;           // first 128-element row of this warp's part of the tile
             uint32_t *const gbase = out32 + size_t(scan_row) * p.scan_pitch + size_t(row0) * kTileCols + piece * 4;
             const int rows_here = int(p.rows128) - int(row0);         // rows of this part that exist (ragged last tile)
@@ -1176,11 +1280,13 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 uint32_t o[32];
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
+                    if (CHUNK_TC && !level0 && ((q * 32 + c) % S) == 0)   // start of a chunk: its carry comes from the product
+                        run = add32<IS_INT>(base, chunk_carry[(q * 32 + c) / S]);
                     uint32_t v = add32<IS_INT>(d[c], run);
                     o[c] = EXCL ? prev : v;
                     prev = v;
                     const bool chunk_end = (S <= 32) ? (((c + 1) % S) == 0) : (c == 31 && (((q + 1) * 32) % S) == 0);
-                    if (chunk_end && !level0) run = v;                // end of a chunk: its total joins the carry
+                    if (!CHUNK_TC && chunk_end && !level0) run = v;   // end of a chunk: its total joins the carry
                 }
                 if (level0 && EXCL) {                                 // not a meaningful combination; keep it defined
 #pragma unroll

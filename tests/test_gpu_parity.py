@@ -188,7 +188,7 @@ def test_row_total_scan_on_tensor_cores_gives_the_same_integers(runner):
     check(runner, np.full(5 * TILE, 127, np.int8), "i8", 16, upper_level_path=1)
     d = torch.zeros(256, dtype=torch.int8, device="cuda")
     o = torch.zeros(256, dtype=torch.int32, device="cuda")
-    assert B.tcu_scan_ex(d, o, 1, 256, 0, 16, runner.ws_ptr, runner.ws_bytes, 0, upper_level_path=2) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_ex(d, o, 1, 256, 0, 16, runner.ws_ptr, runner.ws_bytes, 0, upper_level_path=3) == B.TCU_ERR_INVALID_ARG
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
@@ -206,6 +206,32 @@ def test_row_total_scan_on_tensor_cores_floating_point(runner, dtype):
     assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
     check(runner, gen(dtype, 7 * TILE + 3, 5), dtype, 128, upper_level_path=1, down_sweep_path=1)   # both products at once
     assert runner.stats["upper_level_path"] == 1 and runner.stats["down_sweep_path"] == 1
+
+
+@pytest.mark.parametrize("dtype", ["i8", "f16", "bf16"])
+def test_chunk_level_on_tensor_cores(runner, dtype):
+    # upper_level_path = 2: besides the scan over the row totals, the carries of the 128 / s chunks of a row are a product
+    # of the chunk totals (two 8-bit limbs / three bf16 terms) with a strictly upper triangular ones matrix
+    from tests.gpu_util import check
+    per_tile = {"i8": {16: 4 + 4 + 4 + 1, 64: 4 + 4 + 4 + 1}, "f": {16: 8 + 8 + 8 + 2, 64: 8 + 8 + 8 + 2}}["i8" if dtype == "i8" else "f"]
+    for n, s in [(TILE, 16), (9 * TILE + 128 * 3 + 5, 64), (500 * TILE + 77, 16), (300 * TILE, 64)]:
+        x = gen(dtype, n, 7300 + n % 313)
+        check(runner, x, dtype, s, upper_level_path=2)
+        check(runner, x, dtype, s, True, upper_level_path=2)
+        assert runner.stats["upper_level_path"] == 2
+        assert runner.stats["mma_instructions"] == runner.stats["tiles"] * per_tile[s]
+    if dtype == "i8":
+        check(runner, np.full(5 * TILE, -128, np.int8), "i8", 64, upper_level_path=2)     # chunk totals of -2^13: the limb split at its limit
+        check(runner, np.full(5 * TILE, 127, np.int8), "i8", 64, upper_level_path=2)
+        x = ((np.arange(4 * TILE) * 37 + (np.arange(4 * TILE) // 16) * 11) % 251 - 125).astype(np.int8)   # every chunk different
+        check(runner, x, "i8", 16, upper_level_path=2)
+    else:
+        for s in (16, 64):
+            got = runner.run(np.ones(1 << 22, np.float16), "f16", s, upper_level_path=2)
+            assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
+    check(runner, gen(dtype, 3 * TILE + 9, 5), dtype, 128, upper_level_path=2)     # a row of s = 128 is one chunk: same as 1
+    assert runner.stats["upper_level_path"] == 2
+    check(runner, gen(dtype, 64 * 65536, 6).reshape(64, 65536), dtype, 16, upper_level_path=2)   # batched rows too
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])

@@ -73,7 +73,7 @@ def test_argument_checks_return_before_any_launch(B):
     assert B.tcu_scan_batched(ok_in, ok_out, 4, (1 << 40) + 16, 0, 16, 0, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED   # too large
     # the general call: malformed options are refused, carries belong to single arrays only
     assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, variant=2) == B.TCU_ERR_INVALID_ARG
-    assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, upper_level_path=2) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, upper_level_path=3) == B.TCU_ERR_INVALID_ARG
     assert B.tcu_scan_ex(ok_in, ok_out, 2, 16, 0, 16, ok_ws, ws, d_carry_in=0x9000) == B.TCU_ERR_INVALID_ARG
     assert B.tcu_scan_ex(ok_in, ok_out, 1, 16, 0, 16, ok_ws, ws, d_carry_in=0x9004) == B.TCU_ERR_INVALID_ARG  # 8-byte aligned
     assert B.tcu_scan_ex(ok_in, ok_out, 1, 16, 0, 16, ok_ws, ws, variant=1, d_carry_in=0x9000) == B.TCU_ERR_UNSUPPORTED
