@@ -355,6 +355,55 @@ def wait_counters(args):
     print(json.dumps({"wait_counters": report, "sm_ghz_assumed": ghz}))
 
 
+def run_sharded(args):
+    """One array of 2^n_log2 int8 elements split into contiguous shards, one per rank (strong scaling): every step
+    each rank takes the total of its shard, the totals are all-gathered (8 bytes per rank), each rank sums the totals
+    before its own and scans its shard from that carry (paper Section 2.2 steps 2-4 with one segment per device).
+    With one rank the exchange is a copy.  Prints one JSON line on rank 0."""
+    import torch
+    import torch.distributed as dist
+    from paper_2411_17887_b200 import binding as B
+    from paper_2411_17887_b200 import inputs, sharding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    n = 1 << args.n_log2
+    lo, hi = sharding.shard_elements(n, world, rank)
+    x_local = torch.from_numpy(inputs.int8_uniform((hi - lo,), -127, 127, 3 + 1000 * rank)).cuda()
+    out_local = torch.empty(hi - lo, dtype=torch.int32, device="cuda")
+    job = sharding.ShardedScan(hi - lo, "i8", s=S_TILE)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+    for _ in range(max(args.warmup, 3)):
+        job.scan(x_local, out_local)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        job.scan(x_local, out_local)
+    e1.record()
+    barrier()
+    ms_total = sharding.max_over_ranks(e0.elapsed_time(e1), "cuda")
+    B.check(B.tcu_scan_device_status(job.ws_ptr, torch.cuda.current_stream().cuda_stream))
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        print(json.dumps({"metric": METRIC, "value": n * args.steps / (ms_total * 1e-3), "unit": "elements/s", "n_gpus": world,
+                          "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+                          "scaling": "strong", "vs_baseline": None, "dtype": "i32", "data": "synthetic",
+                          "config": {"workload": f"one array of 2^{args.n_log2} int8 sharded over {world} GPU(s): shard total, "
+                                                 "all-gather of the totals, scan from the carry; 6 B/elt per rank (input read twice)"},
+                          "gpu_launches": 4 * args.steps}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -526,6 +575,8 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 ms_w = Timer(torch).loop(widen, 10)
                 extra["widening_copy_i8_i32_n2p28"] = frac({"us": round(1e3 * ms_w, 2), "GBps": round(5 * n / (ms_w * 1e-3) / 1e9, 1)})
+                ms_t = Timer(torch).loop(lambda: d_out.copy_(d_in), 10)      # the framework's own converting copy, same mix
+                extra["torch_copy_i8_to_i32_n2p28"] = frac({"us": round(1e3 * ms_t, 2), "GBps": round(5 * n / (ms_t * 1e-3) / 1e9, 1)})
                 # the same scans in the two-sweep structure (reduce, scan the totals, scan with every carry known)
                 extra["C3_two_sweep"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, variant=1)[0])
                 extra["f16_n2p28_two_sweep"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, variant=1)[0])
@@ -610,6 +661,8 @@ def main():
     ap.add_argument("--n-log2", type=int, default=28, help="log2 of the array length (28 = the headline workload)")
     ap.add_argument("--profile", action="store_true",
                     help="device-resident loop only (no end-to-end leg, no oracle): the command to wrap in ncu")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one array split over the ranks (strong scaling) instead of one array per rank")
     ap.add_argument("--wait-counters", action="store_true",
                     help="debug build of the library: where each role of the kernel waits, at the headline size")
     ap.add_argument("--fixed-cost", action="store_true",
@@ -621,6 +674,8 @@ def main():
         fixed_cost(args)
     elif args.wait_counters:
         wait_counters(args)
+    elif args.sharded:
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -47,3 +47,22 @@ def scan(x: torch.Tensor, s: int = 16, exclusive: bool = False, out: torch.Tenso
     else:
         B.check(B.tcu_scan_batched(x, out, rows, cols, B.DTYPES[dn], s, int(exclusive), ws.ptr, ws.bytes, stream))
     return out
+
+
+def segmented_scan(x: torch.Tensor, offsets: torch.Tensor, s: int = 16, exclusive: bool = False,
+                   out: torch.Tensor = None) -> torch.Tensor:
+    """Scan every segment x[offsets[k]:offsets[k+1]] of a contiguous 1-D CUDA tensor on its own.  `offsets` is an
+    int64 CUDA tensor, non-decreasing, from 0 to len(x)."""
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 1
+    assert offsets.is_cuda and offsets.dtype == torch.int64 and offsets.is_contiguous() and offsets.numel() >= 1
+    dn = dtype_name(x)
+    n = x.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.int32 if dn == "i8" else torch.float32, device=x.device)
+    ws_bytes = B.tcu_scan_segmented_workspace_bytes(n, B.DTYPES[dn], s)
+    buf = torch.zeros(ws_bytes + 256, dtype=torch.uint8, device=x.device)
+    ptr = buf.data_ptr() + (-buf.data_ptr()) % 256
+    stream = torch.cuda.current_stream().cuda_stream
+    B.check(B.tcu_scan_segmented(x, out, n, offsets, offsets.numel() - 1, B.DTYPES[dn], s, int(exclusive), ptr, ws_bytes, stream))
+    B.check(B.tcu_scan_device_status(ptr, stream))
+    return out

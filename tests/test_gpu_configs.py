@@ -87,3 +87,45 @@ def test_beyond_four_gigabytes_of_output():
     compare_piecewise(got, x, "i8", False)
     got = big.run(x, "i8", 128, exclusive=True)
     compare_piecewise(got, x, "i8", True)
+
+
+def test_segmented_at_the_headline_size():
+    # n = 2^28 int8 cut at random points (mean segment 2^12, some empty segments), in the launch configuration the
+    # benchmark times; every output compared with the oracle's per-segment loop
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    n = 1 << 28
+    x = inputs.make(inputs.CONFIGS["C3"])
+    g = inputs.rng(77)
+    cuts = np.sort(g.integers(0, n + 1, size=n >> 12))
+    off = np.concatenate([[0, 0], cuts, cuts[::1000], [n]]).astype(np.int64)
+    off.sort()
+    d_in = torch.from_numpy(x).cuda()
+    d_out = torch.empty(n, dtype=torch.int32, device="cuda")
+    d_off = torch.from_numpy(off).cuda()
+    ws_bytes = B.tcu_scan_segmented_workspace_bytes(n, B.TCU_I8_I32, 16)
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+    ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+    B.check(B.tcu_scan_workspace_init(ptr, ws_bytes, 0))
+    B.check(B.tcu_scan_segmented(d_in, d_out, n, d_off, off.size - 1, B.TCU_I8_I32, 16, 0, ptr, ws_bytes, 0))
+    B.check(B.tcu_scan_device_status(ptr, 0))
+    got = d_out.cpu().numpy()
+    want = so.scan_segments(x, "i8", off)["y32"]
+    assert np.array_equal(got, want)
+
+
+def test_batched_rows_of_odd_length_at_size():
+    # 4099 rows of 65521 bf16 values (neither a multiple of 16): rows become segments of one 2^28-sized array
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from tests.gpu_util import Runner
+    rows, cols = 4099, 65521
+    x = inputs.bf16_normal((rows, cols), 41)
+    runner = Runner(rows, cols)
+    got = runner.run(x, "bf16", 16, False)
+    assert runner.stats["segments_path"] == 1
+    block = 512
+    for r0 in range(0, rows, block):
+        y, a = so.scan_f64(so.widen(x[r0:r0 + block], "bf16"))
+        err = np.abs(got[r0:r0 + block].astype(np.float64) - y)
+        assert (err <= so.float_tolerance(a)).all(), f"rows {r0}.."
