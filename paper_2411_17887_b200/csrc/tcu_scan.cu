@@ -62,13 +62,13 @@ struct Shape {
     uint64_t rows, cols;
 };
 
-template <bool IS_INT, int S, bool EXCL, bool CHUNK_TC = false>
+template <bool IS_INT, int S, bool EXCL, int VARIANT>
 cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
     static std::atomic<int> configured{-1};
     int dev = 0;
     cudaGetDevice(&dev);
     if (configured.load() != dev) {
-        cudaError_t e = cudaFuncSetAttribute(tcu_scan_kernel<IS_INT, S, EXCL, CHUNK_TC>,
+        cudaError_t e = cudaFuncSetAttribute(tcu_scan_kernel<IS_INT, S, EXCL, VARIANT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
         if (e != cudaSuccess) return e;
         configured.store(dev);
@@ -85,15 +85,25 @@ cudaError_t launch_main(const ScanParams &prm, dim3 grid, size_t smem, cudaStrea
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tcu_scan_kernel<IS_INT, S, EXCL, CHUNK_TC>, prm);
+    return cudaLaunchKernelEx(&cfg, tcu_scan_kernel<IS_INT, S, EXCL, VARIANT>, prm);
+}
+
+// variant: kLean for the plain scan, kFull when any run-time option is in use, kChunk for the chunk-level product
+template <bool IS_INT, int S, bool EXCL>
+cudaError_t dispatch_variant(int variant, const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
+    if constexpr (S < kTileCols) {
+        if (variant == kChunk) return launch_main<IS_INT, S, EXCL, kChunk>(prm, grid, smem, stream);
+    }
+    if (variant != kLean) return launch_main<IS_INT, S, EXCL, kFull>(prm, grid, smem, stream);   // (s = 128: a row is one chunk)
+    return launch_main<IS_INT, S, EXCL, kLean>(prm, grid, smem, stream);
 }
 
 template <bool IS_INT, bool EXCL>
-cudaError_t dispatch_s(int s, bool chunk_tc, const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
+cudaError_t dispatch_s(int s, int variant, const ScanParams &prm, dim3 grid, size_t smem, cudaStream_t stream) {
     switch (s) {
-        case 16: return chunk_tc ? launch_main<IS_INT, 16, EXCL, true>(prm, grid, smem, stream) : launch_main<IS_INT, 16, EXCL>(prm, grid, smem, stream);
-        case 64: return chunk_tc ? launch_main<IS_INT, 64, EXCL, true>(prm, grid, smem, stream) : launch_main<IS_INT, 64, EXCL>(prm, grid, smem, stream);
-        default: return launch_main<IS_INT, 128, EXCL>(prm, grid, smem, stream);   // a row is one chunk: no chunk level
+        case 16: return dispatch_variant<IS_INT, 16, EXCL>(variant, prm, grid, smem, stream);
+        case 64: return dispatch_variant<IS_INT, 64, EXCL>(variant, prm, grid, smem, stream);
+        default: return dispatch_variant<IS_INT, 128, EXCL>(variant, prm, grid, smem, stream);
     }
 }
 
@@ -316,11 +326,15 @@ tcu_status_t scan_impl(const Call &c) {
         }
         dim3 grid(unsigned(tiles < ctas ? tiles : ctas));
         st.grid = grid.x;
+        // the plain scan has a kernel of its own, with every option compiled out
+        const bool plain = !upper_tc && !down_tc && !c.segmented && !level0 && !two_sweep && !c.d_stamps && !c.d_carry_out &&
+                           c.skip_tile == kNoTile;
+        const int variant = chunk_tc ? kChunk : (plain ? kLean : kFull);
         cudaError_t e;
         if (dt == TCU_I8_I32)
-            e = exclusive ? dispatch_s<true, true>(s, chunk_tc, prm, grid, smem, stream) : dispatch_s<true, false>(s, chunk_tc, prm, grid, smem, stream);
+            e = exclusive ? dispatch_s<true, true>(s, variant, prm, grid, smem, stream) : dispatch_s<true, false>(s, variant, prm, grid, smem, stream);
         else
-            e = exclusive ? dispatch_s<false, true>(s, chunk_tc, prm, grid, smem, stream) : dispatch_s<false, false>(s, chunk_tc, prm, grid, smem, stream);
+            e = exclusive ? dispatch_s<false, true>(s, variant, prm, grid, smem, stream) : dispatch_s<false, false>(s, variant, prm, grid, smem, stream);
         if (e != cudaSuccess) return TCU_ERR_CUDA;
     }
     if (c.segmented) {

@@ -68,10 +68,10 @@ constexpr int kChunkNumTot = 4;         // row-total accumulators left when the 
 constexpr int kChunkScratch = kTotBase + kChunkNumTot * kTotCols;    // first TMEM column of the chunk products' results
 constexpr int kEpilogueThreads = 128;
 // Registers per thread after re-allocation.  The pool is what the CTA was launched with (80 x 768 or
-// 96 x 640 = 61440 registers), so 128 x (64 + 64 + 88 + kStoreGroups x kStoreRegs) must not exceed it:
+// 96 x 640 = 61440 registers), so 128 x (64 + 80 + 72 + kStoreGroups x kStoreRegs) must not exceed it:
 // an increase that cannot be granted would block.
 constexpr int kStoreRegs = 128;
-static_assert(128 * (64 + 64 + 88 + kStoreGroups * kStoreRegs) <= 61440, "register pool");
+static_assert(128 * (64 + 80 + 72 + kStoreGroups * kStoreRegs) <= 61440, "register pool");
 constexpr int kFirstStoreWarp = 4;                                   // carry add and store: kStoreGroups x 4 warps
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back (warp 3 is one more)
@@ -420,9 +420,21 @@ __device__ __forceinline__ uint32_t add32(uint32_t a, uint32_t b) {
 }
 
 // ------------------------------------------------------------------------------------ kernel
-template <bool IS_INT, int S, bool EXCL, bool CHUNK_TC = false>
+// VARIANT: kLean = the plain scan (inclusive / exclusive, single array or dense rows, optional carry in): every option
+// below is compiled out; kFull = all run-time options (upper-level and down-sweep products, segments, two-sweep
+// records, level-0 debug output, time stamps, the self-test's silent tile, carry out); kChunk = kFull plus the chunk
+// level as a product.  The plain scan gets a kernel of its own because the options cost it 2-3 % even when they are
+// switched off (measured on 16-bit input: 251 -> 245 µs at n = 2^28, 69.4 -> 67.8 at 2^26, 6.3 -> 5.9 at 2^16) -
+// code size and register allocation of a kernel whose 20 warps run five different programs.
+enum ScanVariant { kLean = 0, kFull = 1, kChunk = 2 };
+template <bool IS_INT, int S, bool EXCL, int VARIANT = kLean>
 __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_constant__ ScanParams p) {
+    constexpr bool FULL = VARIANT != kLean, CHUNK_TC = VARIANT == kChunk;
     static_assert(!CHUNK_TC || S < kTileCols, "a row of s = 128 is one chunk: there is no chunk level");
+    const bool use_upper = FULL && p.upper_tc != 0, use_down = FULL && p.down_tc != 0, segmented = FULL && p.seg_rowflag != nullptr;
+    const bool level0_only = FULL && p.level0_only != 0, prefilled = FULL && p.prefilled != 0, use_stamps = FULL && p.stamps != nullptr;
+    const bool has_carry_out = FULL && p.carry_out != nullptr;
+    const uint32_t skip_tile = FULL ? p.skip_publish_tile : kNoTile;
     constexpr int kTotRing = CHUNK_TC ? kChunkNumTot : kNumTot;   // depth of the ring of row-total accumulators
     using CO = CarryOps<IS_INT>;
     using CarryT = typename CO::T;
@@ -444,11 +456,11 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *in_ring = const_region + p.b_bytes;
     uint8_t *out_ring = in_ring + p.in_stages * kStageBytes;
     uint8_t *seg_ring = out_ring + kOutRingBytes;         // only present for a segmented scan (never together with the two below)
-    uint8_t *upper_a = out_ring + kOutRingBytes;          // only present when p.upper_tc
+    uint8_t *upper_a = out_ring + kOutRingBytes;          // only present when use_upper
     uint8_t *upper_b = upper_a + (IS_INT ? 1 : 2) * kAtomBytes;
-    uint8_t *down_a = upper_a + (p.upper_tc ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present when p.down_tc
+    uint8_t *down_a = upper_a + (use_upper ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present when use_down
     uint8_t *down_b = down_a + kStoreGroups * kAtomBytes;
-    uint8_t *chunk_a = upper_a + (p.upper_tc ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present in the CHUNK_TC variant
+    uint8_t *chunk_a = upper_a + (use_upper ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present in the CHUNK_TC variant
     uint8_t *chunk_b = chunk_a + kStoreGroups * kAtomBytes;
 
     WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
@@ -460,7 +472,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 
     // Optional time stamps (p.stamps is NULL in normal use): each point is passed by one designated thread.
     auto stamp = [&](int k) {
-        if (p.stamps != nullptr) p.stamps[size_t(blockIdx.x) * kStampsPerCta + k] = global_timer_ns();
+        if (use_stamps) p.stamps[size_t(blockIdx.x) * kStampsPerCta + k] = global_timer_ns();
     };
 
     // ---- set-up
@@ -523,14 +535,14 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             st_shared_v4(cbase + (c >> 3) * kAtomBytes + n * 128 + (((c & 7) ^ (n & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
         }
-        if (!IS_INT && p.down_tc) {
+        if (!IS_INT && use_down) {
             // carry operands start as zeros (only 3 of the 16 K-entries of a row are ever written); the other
             // operand is all ones in bf16
             for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 16; e += kThreads) st_shared_v4(smem_u32(down_a) + e * 16, 0u, 0u, 0u, 0u);
             for (int e = threadIdx.x; e < kAtomBytes / 16; e += kThreads)
                 st_shared_v4(smem_u32(down_b) + e * 16, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
         }
-        if (p.upper_tc) {
+        if (use_upper) {
             // A[m][k] = 1 for k < m: its product with a column of row totals is their exclusive scan over the rows
             // (int8 ones for integer scans, bf16 ones otherwise: 16 or 8 K entries per 16-byte piece)
             constexpr int kUpPerPiece = IS_INT ? 16 : 8;
@@ -702,14 +714,14 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 }
                 // publish even after a give-up so that successors do not wait for this tile (a tile in which a
                 // segment starts has already published its final record)
-                if (lane == 0 && !p.prefilled && t != p.skip_publish_tile && !(p.seg_rowflag != nullptr && ctl->agg_cut[ts]))
+                if (lane == 0 && !prefilled && t != skip_tile && !(segmented && ctl->agg_cut[ts]))
                     st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | kStatusInclusive, CO::enc(prefix + agg));
             }
             if (lane == 0) {
                 TRACE(t, 5);
                 ctl->carry_slot[ts] = CO::enc(prefix);
                 mbar_arrive(smem_u32(&ctl->carry_ready[ts]));
-                if (p.carry_out != nullptr && t + 1 == p.tiles_total) *reinterpret_cast<uint64_t *>(p.carry_out) = CO::enc(prefix + agg);
+                if (has_carry_out && t + 1 == p.tiles_total) *reinterpret_cast<uint64_t *>(p.carry_out) = CO::enc(prefix + agg);
                 if (j == 0) stamp(kStampCarry);
             }
             __syncwarp();
@@ -756,7 +768,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     continue;
                 }
                 TRACE(t, 0);
-                const bool seg = p.seg_rowflag != nullptr;
+                const bool seg = segmented;
                 mbar_expect_tx(bar, kStageBytes + (seg ? kSegNoteBytes : 0));
                 if (seg) {
                     // the notes about the tile's rows travel with the tile: two bulk copies that complete on the
@@ -893,10 +905,10 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         lookback_role(0);
     }
     } else if (warp >= kFirstLookbackWarp) {
-        reg_dec<64>();
+        reg_dec<80>();
         lookback_role(uint32_t(warp - kFirstLookbackWarp + 1));
     } else if (warp >= kFirstTotalsWarp) {
-        reg_dec<88>();
+        reg_dec<72>();
         // ------------------------------------------------------------------ totals (up-sweep above the product)
         // Takes the 128 row totals from the small accumulator, scans them across the rows, and
         // publishes the tile total - as soon as the tile has landed, so that the cross-tile look-back
@@ -927,7 +939,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             if (r == 0) TRACE(t, 2);
             uint32_t seg_fl = 0, seg_rv = 0;                          // segmented scan: this row's notes
-            if (p.seg_rowflag != nullptr) {
+            if (segmented) {
                 // the notes of the tile's 128 rows came in with the tile (bulk copies issued by the producer)
                 const uint8_t *notes = seg_ring + ts * kSegNoteBytes;
                 seg_fl = notes[r];
@@ -936,7 +948,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             tc_fence_after();
             const uint32_t rowtot = tmem_ld1(lane_base + kTotBase + tt * kTotCols);
             tmem_ld_wait();
-            if (p.upper_tc) {
+            if (use_upper) {
                 // Paper-faithful variant of this level: the scan over the 128 row totals is itself a product
                 // with a triangular all-ones matrix, D[m][n] = sum over k < m of term n of total k.  Row totals
                 // are int32 / fp32, not tensor-core input types, so each is first split exactly into narrow
@@ -1003,7 +1015,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     const CarryT a = IS_INT ? CarryT(tile_total) : CarryT(__uint_as_float(tile_total));
                     const bool first = (t % p.tiles_per_row == 0);
                     const uint32_t status = first ? kStatusInclusive : kStatusPartial;
-                    if (!p.prefilled && t != p.skip_publish_tile)
+                    if (!prefilled && t != skip_tile)
                         st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
                     ctl->agg_slot[ts] = CO::enc(a);
                 }
@@ -1013,7 +1025,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&ctl->tot_empty[tt]));                // the small accumulator may be refilled
-            if (p.seg_rowflag == nullptr) {
+            if (!segmented) {
                 // ordinary scan: inclusive prefix sums of the row totals across the warp's 32 rows, one hop through
                 // shared memory across the four warps
                 uint32_t inc = rowtot;
@@ -1039,7 +1051,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                     // the first tile of a scan has nothing before it: its total is already inclusive
                     const bool first = (t % p.tiles_per_row == 0);
                     const uint32_t status = first ? kStatusInclusive : kStatusPartial;
-                    if (!p.prefilled && t != p.skip_publish_tile)
+                    if (!prefilled && t != skip_tile)
                         st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc(first ? a + carry_in : a));
                     TRACE(t, 3);
                     if (j == 0) stamp(kStampPublished);
@@ -1115,7 +1127,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 // only what follows that start: in both cases its total is final at once
                 const bool first = (t % p.tiles_per_row == 0);
                 const uint32_t status = (first || run_cut) ? kStatusInclusive : kStatusPartial;
-                if (!p.prefilled && t != p.skip_publish_tile)
+                if (!prefilled && t != skip_tile)
                     st_record(records + size_t(t) * 16, (uint64_t(epoch) << 2) | status, CO::enc((first && !run_cut) ? a + carry_in : a));
                 TRACE(t, 3);
                 if (j == 0) stamp(kStampPublished);
@@ -1144,7 +1156,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         // The carry-product variant makes the four warps of a group meet at a barrier inside the loop, so
         // there they must also leave the loop together: the outcome of every wait is then voted on by the
         // whole group.  In the default path a warp shares no barrier with the others and votes alone.
-        const bool carry_product = !IS_INT && S == 128 && p.down_tc && !p.level0_only;
+        const bool carry_product = !IS_INT && S == 128 && use_down && !level0_only;
         const bool group_meets = carry_product || CHUNK_TC;       // (the chunk product has the same group barrier)
         auto gave_up = [&](bool ok) {
             return group_meets ? named_barrier_or(3 + group, kEpilogueThreads, !ok) : !__all_sync(0xffffffffu, ok);
@@ -1169,12 +1181,12 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             {
                 CarryT carry = CO::dec(ctl->carry_slot[ts]);
                 // segmented scan: a segment starts before this row, inside the tile
-                if (p.seg_rowflag != nullptr && ((ctl->seg_cut[ts][wq] >> lane) & 1u)) carry = CarryT(0);
+                if (segmented && ((ctl->seg_cut[ts][wq] >> lane) & 1u)) carry = CarryT(0);
                 uint32_t rp = rowpref[ts * kTileRows + r];
                 if (IS_INT) base = uint32_t(carry) + rp;
                 else base = __float_as_uint(static_cast<float>(double(carry) + double(__uint_as_float(rp))));
             }
-            const bool level0 = p.level0_only != 0;
+            const bool level0 = level0_only;
             if (level0) base = 0;
             uint32_t run = base;                                      // sum of everything before the current chunk
             uint32_t prev = base;                                     // value of the element to the left (exclusive form)
@@ -1326,7 +1338,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             mbar_arrive(smem_u32(&ctl->ring_free[ts]));
         }
         if (lane == 0 && wq == 0) PROF_FLUSH(32 + 8 * group, 6);
-        if (lane == 0 && wq == 0 && p.stamps != nullptr) p.stamps[size_t(blockIdx.x) * kStampsPerCta + kStampTiles + group] = stored;
+        if (lane == 0 && wq == 0 && use_stamps) p.stamps[size_t(blockIdx.x) * kStampsPerCta + kStampTiles + group] = stored;
     }
 
     // ---- tear-down
