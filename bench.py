@@ -567,14 +567,21 @@ def run_ours(args):
                 extra["C4_4096x65536_bf16"] = frac(time_extra(B, torch, xb, 4096, 65536, 2, 16, ws_ptr, ws_bytes)[0])
                 del xb
                 extra["C1_n2p16_i8"] = time_extra(B, torch, d_in, 1, 1 << 16, 0, 16, ws_ptr, ws_bytes, reps=200)[0]
-                # a plain widening copy with the same 1 : 4 read / write mix, for what that mix reaches without a scan
-                def widen():
-                    B.check(B.tcu_widen_copy_i8_i32(d_in, d_out, n, stream))
-                for _ in range(3):
-                    widen()
-                torch.cuda.synchronize()
-                ms_w = Timer(torch).loop(widen, 10)
-                extra["widening_copy_i8_i32_n2p28"] = frac({"us": round(1e3 * ms_w, 2), "GBps": round(5 * n / (ms_w * 1e-3) / 1e9, 1)})
+                # plain widening copies with the scans' read / write mixes (1 : 4 and 2 : 4), no dependence between
+                # elements: what the memory system gives that mix when nothing has to be carried along
+                d_out_f = d_out.view(torch.float32)
+                for key, src, dst, dtc, bpe in (("widening_copy_i8_i32_n2p28", d_in, d_out, 0, 5),
+                                                ("widening_copy_f16_f32_n2p28", xf, d_out_f, 1, 6)):
+                    def widen():
+                        B.check(B.tcu_widen_copy(src, dst, n, dtc, stream))
+                    for _ in range(3):
+                        widen()
+                    torch.cuda.synchronize()
+                    ms_w = Timer(torch).loop(widen, 20)
+                    extra[key] = frac({"us": round(1e3 * ms_w, 2), "GBps": round(bpe * n / (ms_w * 1e-3) / 1e9, 1)})
+                line["config"]["scan_time_over_widening_copy_time"] = {
+                    "i8": round(1e3 * ms_step / extra["widening_copy_i8_i32_n2p28"]["us"], 4),
+                    "f16": round(line["config"]["fp16_n2p28_s16"]["us"] / extra["widening_copy_f16_f32_n2p28"]["us"], 4)}
                 ms_t = Timer(torch).loop(lambda: d_out.copy_(d_in), 10)      # the framework's own converting copy, same mix
                 extra["torch_copy_i8_to_i32_n2p28"] = frac({"us": round(1e3 * ms_t, 2), "GBps": round(5 * n / (ms_t * 1e-3) / 1e9, 1)})
                 # the same scans in the two-sweep structure (reduce, scan the totals, scan with every carry known)

@@ -278,10 +278,14 @@ size_t tcu_sort_tmp_bytes(size_t n);
 tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_t n, void *d_tmp, size_t tmp_bytes,
                           void *d_ws, size_t ws_bytes, cudaStream_t stream);
 
-/* Measuring aid (no counterpart in the paper): out[i] = in[i] widened from int8 to int32, a plain copy kernel with the
- * traffic mix of the int8 scan (1 byte read, 4 bytes written per element).  The benchmark times it beside the scan
- * to show what that mix reaches on the machine's memory system.  n a multiple of 16, both pointers 16-byte aligned. */
-tcu_status_t tcu_widen_copy_i8_i32(const void *d_in, void *d_out, size_t n, cudaStream_t stream);
+/* Measuring aid (no counterpart in the paper): out[i] = in[i] widened to the output type of `dt` (int8 -> int32,
+ * fp16 / bf16 -> fp32, all exact), a plain copy kernel with the traffic mix of the scan of that type (1 or 2 bytes
+ * read, 4 bytes written per element) and no dependence between elements.  The benchmark times it beside the scan to
+ * show what that mix reaches on the machine's memory system.
+ *   d_in, d_out   device pointers, 16-byte aligned, not overlapping; n elements, n a multiple of 4
+ * Errors: TCU_ERR_INVALID_ARG (null or misaligned pointer, n not a multiple of 4, unknown dt), TCU_ERR_UNSUPPORTED
+ * (n >= 2^42), TCU_ERR_CUDA (the launch failed).  Asynchronous on `stream`. */
+tcu_status_t tcu_widen_copy(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, cudaStream_t stream);
 
 /* Copies the bookkeeping of the most recent scan call made by the calling thread. */
 tcu_status_t tcu_scan_last_stats(tcu_scan_stats_t *out);

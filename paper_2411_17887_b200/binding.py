@@ -83,8 +83,8 @@ _lib.tcu_sort_tmp_bytes.argtypes = [_sz]
 _lib.tcu_sort_tmp_bytes.restype = _sz
 _lib.tcu_sort_u32.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _sz, _vp]
 _lib.tcu_sort_u32.restype = _int
-_lib.tcu_widen_copy_i8_i32.argtypes = [_vp, _vp, _sz, _vp]
-_lib.tcu_widen_copy_i8_i32.restype = _int
+_lib.tcu_widen_copy.argtypes = [_vp, _vp, _sz, _int, _vp]
+_lib.tcu_widen_copy.restype = _int
 _lib.tcu_scan_last_stats.argtypes = [ctypes.POINTER(TcuScanStats)]
 _lib.tcu_scan_last_stats.restype = _int
 _lib.tcu_status_string.argtypes = [_int]
@@ -201,8 +201,8 @@ def tcu_sort_u32(d_keys_in, d_keys_out, n: int, d_tmp, tmp_bytes: int, d_ws, ws_
     return _lib.tcu_sort_u32(_p(d_keys_in), _p(d_keys_out), n, _p(d_tmp), tmp_bytes, _p(d_ws), ws_bytes, stream)
 
 
-def tcu_widen_copy_i8_i32(d_in, d_out, n: int, stream=0) -> int:
-    return _lib.tcu_widen_copy_i8_i32(_p(d_in), _p(d_out), n, stream)
+def tcu_widen_copy(d_in, d_out, n: int, dt: int, stream=0) -> int:
+    return _lib.tcu_widen_copy(_p(d_in), _p(d_out), n, dt, stream)
 
 
 def tcu_scan_last_stats() -> dict:

@@ -701,14 +701,17 @@ tcu_status_t tcu_sort_u32(const uint32_t *d_keys_in, uint32_t *d_keys_out, size_
     return TCU_OK;
 }
 
-tcu_status_t tcu_widen_copy_i8_i32(const void *d_in, void *d_out, size_t n, cudaStream_t stream) {
+tcu_status_t tcu_widen_copy(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, cudaStream_t stream) {
+    if (dt != TCU_I8_I32 && dt != TCU_F16_F32 && dt != TCU_BF16_F32) return TCU_ERR_INVALID_ARG;
     if (n == 0) return TCU_OK;
-    if (!d_in || !d_out || (n % 16) != 0) return TCU_ERR_INVALID_ARG;
+    if (!d_in || !d_out || (n % 4) != 0) return TCU_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(d_in) & 15) || (reinterpret_cast<uintptr_t>(d_out) & 15)) return TCU_ERR_INVALID_ARG;
-    int sms = sm_count();
-    if (sms <= 0) return TCU_ERR_CUDA;
-    tcu_widen_copy_kernel<<<unsigned(sms) * 8, 256, 0, stream>>>(reinterpret_cast<const int4 *>(d_in), reinterpret_cast<int4 *>(d_out),
-                                                                uint64_t(n / 16));
+    const uint64_t pieces = n / 4, per_block = uint64_t(kWidenThreads) * kWidenPerThread;
+    const uint64_t blocks = (pieces + per_block - 1) / per_block;
+    if (blocks >= (1ull << 31)) return TCU_ERR_UNSUPPORTED;
+    if (dt == TCU_I8_I32) tcu_widen_copy_kernel<0><<<unsigned(blocks), kWidenThreads, 0, stream>>>(d_in, d_out, pieces);
+    else if (dt == TCU_F16_F32) tcu_widen_copy_kernel<1><<<unsigned(blocks), kWidenThreads, 0, stream>>>(d_in, d_out, pieces);
+    else tcu_widen_copy_kernel<2><<<unsigned(blocks), kWidenThreads, 0, stream>>>(d_in, d_out, pieces);
     return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
 }
 

@@ -76,6 +76,7 @@ constexpr int kFirstStoreWarp = 4;                                   // carry ad
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back (warp 3 is one more)
 constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps - 1);
+constexpr int kEpochThread = 2 * 32;     // lane 0 of warp 2: reads the epoch of a launch whose CTAs have one tile each
 // The register re-allocation below assumes that the kernel is compiled at 96 registers per thread, which is what
 // 640 threads per CTA give.  With more threads the compiler settles on fewer (80 at 672), and a setmaxnreg.dec to a
 // value above the current allocation is an illegal instruction: do not add warps without redoing the numbers.
@@ -476,6 +477,18 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     };
 
     // ---- set-up
+    if (threadIdx.x == kThreads - 1 && kPrefetchDist > 0) {
+        // The producers prefetch tile t + kPrefetchDist into L2 when they claim tile t, which leaves the first
+        // kPrefetchDist tiles of the launch to nobody: start their trip from DRAM now, before the set-up, the wait
+        // for the previous kernel and the first ticket (a prefetch moves data into L2, the point of coherence, so it
+        // may run ahead of a previous kernel that is still writing the input).
+        for (uint32_t tp = blockIdx.x; tp < kPrefetchDist && tp < p.tiles_total; tp += gridDim.x) {
+            const int prow = tp / p.tiles_per_row, plt = tp % p.tiles_per_row;
+#pragma unroll
+            for (int a = 0; a < kInAtoms; ++a)
+                tma_prefetch_l2_3d(&p.tmap_in, a * (128 / kElemBytes), plt * kTileRows, prow);
+        }
+    }
     if (threadIdx.x == 0) {
         stamp(kStampEntry);
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&p.tmap_in)) : "memory");
@@ -599,9 +612,14 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     Waiter w{ctl, hdr, p.spin_limit};
     uint32_t first_ticket = 0;                 // (thread 0 only) first tile of this CTA
     uint32_t my_epoch = 0;                     // (thread 0 only) the epoch of this launch
-    if (threadIdx.x == 0) {
-        stamp(kStampDepsDone);
-        first_ticket = atomicAdd(&hdr->ticket, 1u);
+    // A launch with no more tiles than CTAs hands tile b to CTA b - nothing to claim, no round trip to the workspace
+    // before the first load - and lets a thread that is idle until the tile lands fetch the epoch.  (With several
+    // tiles per CTA the first one is claimed like the others: a CTA that starts late - behind the tail of the
+    // previous kernel, say - must not sit on an early tile.)
+    const bool single_wave = p.tiles_total <= gridDim.x;
+    if (threadIdx.x == 0) stamp(kStampDepsDone);
+    if (threadIdx.x == (single_wave ? kEpochThread : 0)) {
+        first_ticket = single_wave ? 0u : atomicAdd(&hdr->ticket, 1u);
         my_epoch = ld_relaxed_u32(&hdr->epoch) + 1;
         ctl->epoch = my_epoch;
         // what precedes the whole scan (continuation of an earlier piece or shard); only single-array calls pass one
@@ -756,7 +774,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
                 PROF_ADD(0);
                 uint32_t t = kNoTile;
-                if (markers == 0) t = (j == 0) ? first_ticket : atomicAdd(&hdr->ticket, 1u);
+                if (markers == 0) t = single_wave ? (j == 0 ? blockIdx.x : kNoTile) : (j == 0 ? first_ticket : atomicAdd(&hdr->ticket, 1u));
                 if (t >= p.tiles_total) t = kNoTile;
                 PROF_ADD(1);
                 PROF_INC(3, 1);
@@ -803,6 +821,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             // again (records are compared with the copy of the epoch in shared memory), and the next launch
             // reads them only after this one has completed.  Doing it here, not at the end of the CTA, keeps
             // the round trip of the atomic off the tail of the kernel.
+            if (single_wave && w.wait(smem_u32(&ctl->epoch_ready), 0)) my_epoch = ctl->epoch;
             {
                 const uint32_t arrived = atomicAdd(&hdr->done, 1u);
                 if (arrived == gridDim.x - 1) {
@@ -1674,20 +1693,53 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
     }
 }
 
-// ---- measuring aid: a plain widening copy with the scan's traffic mix (1 byte read, 4 bytes written per element), to
-// see what that mix reaches on this memory system without any scan in the way
-__global__ void __launch_bounds__(256) tcu_widen_copy_kernel(const int4 *in, int4 *out, uint64_t pieces) {
-    for (uint64_t i = uint64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < pieces; i += uint64_t(gridDim.x) * blockDim.x) {
-        const int4 v = in[i];                     // 16 int8 values
-        const int w[4] = {v.x, v.y, v.z, v.w};
+// ---- measuring aid: a plain widening copy with the scan's traffic mix (1 or 2 bytes read, 4 bytes written per
+// element), to see what that mix reaches on this memory system without any scan in the way.  Every thread reads
+// kWidenPerThread pieces of four elements and writes each as one 16-byte store, so that a warp reads whole 128-byte
+// (or 256-byte) runs and writes whole 512-byte runs; one piece of the array per block, no loop over the grid (the
+// fastest of the block sizes and unroll factors tried: persistent grids and one piece per thread were 10-30 % slower).
+constexpr int kWidenThreads = 256;
+constexpr int kWidenPerThread = 2;
+template <int DTYPE>
+__global__ void __launch_bounds__(kWidenThreads) tcu_widen_copy_kernel(const void *__restrict__ in, void *__restrict__ out, uint64_t pieces) {
+    const uint64_t base = uint64_t(blockIdx.x) * (kWidenThreads * kWidenPerThread) + threadIdx.x;
+    if (DTYPE == 0) {
+        uint32_t w[kWidenPerThread];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < kWidenPerThread; ++k) {
+            const uint64_t i = base + k * kWidenThreads;
+            w[k] = i < pieces ? reinterpret_cast<const uint32_t *>(in)[i] : 0u;
+        }
+#pragma unroll
+        for (int k = 0; k < kWidenPerThread; ++k) {
+            const uint64_t i = base + k * kWidenThreads;
             int4 o;
             o.x = int(int8_t(w[k] & 0xFF));
             o.y = int(int8_t((w[k] >> 8) & 0xFF));
             o.z = int(int8_t((w[k] >> 16) & 0xFF));
-            o.w = int(int8_t((w[k] >> 24) & 0xFF));
-            out[4 * i + k] = o;
+            o.w = int(int8_t(w[k] >> 24));
+            if (i < pieces) reinterpret_cast<int4 *>(out)[i] = o;
+        }
+    } else {
+        uint2 w[kWidenPerThread];
+#pragma unroll
+        for (int k = 0; k < kWidenPerThread; ++k) {
+            const uint64_t i = base + k * kWidenThreads;
+            w[k] = i < pieces ? reinterpret_cast<const uint2 *>(in)[i] : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int k = 0; k < kWidenPerThread; ++k) {
+            const uint64_t i = base + k * kWidenThreads;
+            float4 o;
+            if (DTYPE == 1) {
+                const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&w[k].x));
+                const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&w[k].y));
+                o = make_float4(a.x, a.y, b.x, b.y);
+            } else {                                  // bf16: the upper half of the fp32 pattern
+                o = make_float4(__uint_as_float(w[k].x << 16), __uint_as_float(w[k].x & 0xFFFF0000u),
+                                __uint_as_float(w[k].y << 16), __uint_as_float(w[k].y & 0xFFFF0000u));
+            }
+            if (i < pieces) reinterpret_cast<float4 *>(out)[i] = o;
         }
     }
 }

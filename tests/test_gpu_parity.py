@@ -255,12 +255,23 @@ def test_widening_copy_measuring_aid():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2411_17887_b200 import binding as B
-    x = gen("i8", 5 * TILE + 16, 77)
-    d_in = torch.from_numpy(x).cuda()
-    d_out = torch.zeros(x.size, dtype=torch.int32, device="cuda")
-    B.check(B.tcu_widen_copy_i8_i32(d_in, d_out, x.size, 0))
-    assert np.array_equal(d_out.cpu().numpy(), x.astype(np.int32))
-    assert B.tcu_widen_copy_i8_i32(d_in, d_out, 17, 0) == B.TCU_ERR_INVALID_ARG
+    from tests.gpu_util import to_device
+    from oracle import scan_oracle as so
+    for dtype in ("i8", "f16", "bf16"):
+        for n in (5 * TILE + 16, 4, 2048, 2052, 3 * 2048 - 4):       # whole blocks, a ragged last block, one piece
+            x = gen(dtype, n, 77)
+            d_in = to_device(x, dtype)
+            d_out = torch.full((n + 8,), 7, dtype=torch.int32 if dtype == "i8" else torch.float32, device="cuda")
+            B.check(B.tcu_widen_copy(d_in, d_out, n, B.DTYPES[dtype], 0))
+            got = d_out.cpu().numpy()
+            want = x.astype(np.int32) if dtype == "i8" else so.widen(x, dtype).astype(np.float32)
+            assert np.array_equal(got[:n], want) and (got[n:] == 7).all()
+    d_in = torch.zeros(64, dtype=torch.int8, device="cuda")
+    d_out = torch.zeros(64, dtype=torch.int32, device="cuda")
+    assert B.tcu_widen_copy(d_in, d_out, 17, 0, 0) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_widen_copy(d_in, d_out, 16, 5, 0) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_widen_copy(d_in[1:], d_out, 16, 0, 0) == B.TCU_ERR_INVALID_ARG
+    assert B.tcu_widen_copy(d_in, d_out, 0, 0, 0) == B.TCU_OK
 
 
 def test_many_back_to_back_launches_agree(runner):
