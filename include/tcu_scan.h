@@ -246,10 +246,12 @@ tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream);
  * returns.  After the stream has drained, tcu_scan_device_status(d_ws) returns TCU_ERR_TIMEOUT,
  * the output is not valid, and the context is still usable; tcu_scan_workspace_init() clears
  * the condition.  Nothing faults or hangs.  skip_tile must be below the number of tiles, and
- * n a multiple of 128. */
+ * n a multiple of 128.  upper_level_path / down_sweep_path select the same optional tensor-core
+ * branches as in tcu_scan_options_t (0 / 0: the ordinary path), whose store and totals warps meet
+ * at barriers inside their loops and must therefore give up together. */
 tcu_status_t tcu_scan_selftest_timeout(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
-                                       size_t skip_tile, unsigned limit_ms,
-                                       void *d_ws, size_t ws_bytes, cudaStream_t stream);
+                                       size_t skip_tile, unsigned limit_ms, int upper_level_path,
+                                       int down_sweep_path, void *d_ws, size_t ws_bytes, cudaStream_t stream);
 
 /* One array split over several devices (paper Section 2.2 steps 2-4 with one segment per device,
  * and the p-TCU bound of its last paragraph): each device computes the total of its shard

@@ -64,7 +64,7 @@ _lib.tcu_scan_host.argtypes = [_vp, _vp, _sz, _int, _int, _int, _vp, _vp, _vp, _
 _lib.tcu_scan_host.restype = _int
 _lib.tcu_scan_device_status.argtypes = [_vp, _vp]
 _lib.tcu_scan_device_status.restype = _int
-_lib.tcu_scan_selftest_timeout.argtypes = [_vp, _vp, _sz, _int, _int, _sz, ctypes.c_uint, _vp, _sz, _vp]
+_lib.tcu_scan_selftest_timeout.argtypes = [_vp, _vp, _sz, _int, _int, _sz, ctypes.c_uint, _int, _int, _vp, _sz, _vp]
 _lib.tcu_scan_selftest_timeout.restype = _int
 _lib.tcu_scan_noalloc_status.argtypes = [_vp]
 _lib.tcu_scan_noalloc_status.restype = _int
@@ -188,9 +188,9 @@ def tcu_scan_device_status(d_ws, stream=0) -> int:
 
 
 def tcu_scan_selftest_timeout(d_in, d_out, n: int, dt: int, s: int, skip_tile: int, limit_ms: int, d_ws,
-                              ws_bytes: int, stream=0) -> int:
-    return _lib.tcu_scan_selftest_timeout(_p(d_in), _p(d_out), n, dt, s, int(skip_tile), int(limit_ms), _p(d_ws),
-                                          ws_bytes, stream)
+                              ws_bytes: int, stream=0, *, upper_level_path: int = 0, down_sweep_path: int = 0) -> int:
+    return _lib.tcu_scan_selftest_timeout(_p(d_in), _p(d_out), n, dt, s, int(skip_tile), int(limit_ms),
+                                          int(upper_level_path), int(down_sweep_path), _p(d_ws), ws_bytes, stream)
 
 
 def tcu_sort_tmp_bytes(n: int) -> int:

@@ -618,10 +618,13 @@ tcu_status_t tcu_scan_device_status(const void *d_ws, cudaStream_t stream) {
 }
 
 tcu_status_t tcu_scan_selftest_timeout(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s, size_t skip_tile,
-                                       unsigned limit_ms, void *d_ws, size_t ws_bytes, cudaStream_t stream) {
+                                       unsigned limit_ms, int upper_level_path, int down_sweep_path, void *d_ws,
+                                       size_t ws_bytes, cudaStream_t stream) {
     if (limit_ms == 0 || limit_ms > 1000) return TCU_ERR_INVALID_ARG;
     if (n == 0 || n % kTileCols != 0 || skip_tile >= tiles_for(1, n)) return TCU_ERR_INVALID_ARG;
     Call c = make_call(d_in, d_out, 1, n, dt, s, false, d_ws, ws_bytes, stream);
+    c.upper_path = upper_level_path;           // (range-checked with the other arguments)
+    c.down_path = down_sweep_path;
     c.skip_tile = uint32_t(skip_tile);
     c.spin_limit = (long long)limit_ms * 2000000LL;            // about 2 cycles per nanosecond
     return scan_impl(c);

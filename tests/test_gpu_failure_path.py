@@ -13,8 +13,16 @@ pytestmark = pytest.mark.gpu
 TILE = 128 * 128
 
 
-@pytest.mark.parametrize("dtype,s,tiles,skip", [("i8", 16, 40, 3), ("f16", 128, 12, 0), ("i8", 64, 400, 150)])
-def test_real_kernel_wait_runs_out_and_recovers(dtype, s, tiles, skip):
+# (input type, s, tiles, silent tile, upper_level_path, down_sweep_path): the ordinary path with the silent tile first,
+# inside the first wave and in the second wave; then the optional tensor-core branches, in which the four totals warps
+# and the four warps of a store group meet at barriers inside their loops and have to give up together
+CASES = [("i8", 16, 40, 3, 0, 0), ("f16", 128, 12, 0, 0, 0), ("i8", 64, 400, 150, 0, 0),
+         ("i8", 16, 40, 3, 1, 0), ("f16", 16, 200, 160, 1, 0), ("f16", 128, 40, 3, 0, 1), ("f16", 128, 300, 149, 1, 1),
+         ("i8", 16, 40, 3, 2, 0), ("f16", 64, 200, 155, 2, 0)]
+
+
+@pytest.mark.parametrize("dtype,s,tiles,skip,upper,down", CASES)
+def test_real_kernel_wait_runs_out_and_recovers(dtype, s, tiles, skip, upper, down):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from oracle import scan_oracle as so
@@ -32,8 +40,10 @@ def test_real_kernel_wait_runs_out_and_recovers(dtype, s, tiles, skip):
     assert B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, skip, 0, ptr, ws_bytes, 0) == B.TCU_ERR_INVALID_ARG
     assert B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, tiles, 20, ptr, ws_bytes, 0) == B.TCU_ERR_INVALID_ARG
     # tile `skip` never publishes; every wait gives up after 20 ms
-    B.check(B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, skip, 20, ptr, ws_bytes, 0))
+    B.check(B.tcu_scan_selftest_timeout(d_in, d_out, n, dt, s, skip, 20, ptr, ws_bytes, 0, upper_level_path=upper,
+                                        down_sweep_path=down))
     assert B.tcu_scan_device_status(ptr, 0) == B.TCU_ERR_TIMEOUT
+    assert B.tcu_scan_last_stats()["upper_level_path"] == upper and B.tcu_scan_last_stats()["down_sweep_path"] == down
     # the tiles before the silent one were not affected
     ref = so.scan(x, dtype)
     got = d_out.cpu().numpy()
