@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes read / input bytes, and bytes the SMs wrote to L2 / output bytes.  DRAM *write* bytes of a capture are
 # not used: tens of MB of the output are still dirty in L2 when the kernel ends, a constant that does not grow with n.
 NCU_READ_RATIO = 1.002
-NCU_WRITE_RATIO = 1.005
+NCU_WRITE_RATIO = 1.004
 
 
 def measured_peak():

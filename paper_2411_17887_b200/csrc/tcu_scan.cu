@@ -245,11 +245,11 @@ tcu_status_t scan_impl(const Call &c) {
     st.segments_path = c.segmented ? 1 : 0;
 
     // segmented scan: note, for every row of 128 elements that holds a segment start, whether it starts the row
-    // and what the row hands on (one warp per start), before the tile kernel runs
+    // and what the row hands on (eight lanes per start), before the tile kernel runs
     uint8_t *seg_flag = nullptr;
     uint32_t *seg_val = nullptr;
     SegSource seg{c.d_offsets, c.seg_pitch, c.num_segments};
-    const unsigned seg_blocks = unsigned((c.num_segments * 32 + 255) / 256);
+    const unsigned seg_blocks = unsigned((c.num_segments * kSegLanes + 255) / 256);
     if (c.segmented) {
         seg_flag = reinterpret_cast<uint8_t *>(d_ws) + seg_flag_offset(cols);
         seg_val = reinterpret_cast<uint32_t *>(reinterpret_cast<uint8_t *>(d_ws) + seg_val_offset(cols));

@@ -1531,7 +1531,7 @@ __global__ void __launch_bounds__(1024) tcu_totals_scan_kernel(void *ws, uint32_
 // one segment and goes through the tensor-core path unchanged.  A row that holds starts is summarised for that path
 // by two values: whether a segment starts at its first element (then nothing carries into the row) and the sum from
 // its last start to its end (what the row hands on).  The elements of such a row from its first start on - the
-// ones the carry of the earlier rows must not reach - are scanned again here, by one warp, straight from the input.
+// ones the carry of the earlier rows must not reach - are scanned again here, by eight lanes, straight from the input.
 
 struct SegSource {
     const uint64_t *offsets;   // num_segments + 1 values, or NULL for equal segments of `pitch` elements
@@ -1542,71 +1542,86 @@ struct SegSource {
 
 enum SegMode { kSegPrepare = 0, kSegFixup = 1, kSegTail = 2 };
 
-// One warp per segment start (modes prepare / fixup; the warp of the first start in a row does the row) or one warp
-// in all (mode tail: the incomplete row at the end of the array, which the tile kernel never stores).
+// kSegLanes lanes per segment start (modes prepare / fixup; the lanes of the first start in a row do the row; a warp
+// works on 32 / kSegLanes starts at once, which is what hides the latency of the offset -> row -> store chain of each)
+// or one such group in all (mode tail: the incomplete row at the end of the array, which the tile kernel never
+// stores).  Every lane holds kSegPerLane consecutive elements of the row.
+constexpr int kSegLanes = 8;
+constexpr int kSegPerLane = kTileCols / kSegLanes;          // 16
 template <bool IS_INT, bool EXCL, int MODE>
 __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, void *out, uint64_t n, SegSource seg, const void *ws,
                                                                uint32_t tiles, uint8_t *rowflag, uint32_t *rowval, uint32_t dtype) {
     using CO = CarryOps<IS_INT>;
     using CarryT = typename CO::T;
     using ValT = typename std::conditional<IS_INT, uint32_t, float>::type;
-    const int lane = threadIdx.x & 31;
+    constexpr unsigned kFull = 0xffffffffu;
+    const int sl = threadIdx.x & (kSegLanes - 1);          // lane within the group of this start
     const uint64_t rows128 = n / kTileCols;
-    uint64_t row, k0;                      // the row this warp handles, and the first segment start inside it
-    bool has_start = true;
+    uint64_t row = 0, k0 = 0;              // the row this group handles, and the first segment start inside it
+    // A group with nothing to do stays in the code (the shuffles below are warp-wide) but touches no memory.
+    bool active = true, has_start = true;
     if (MODE == kSegTail) {
+        active = threadIdx.x < kSegLanes;
         row = rows128;
         // first start at or after the beginning of the row (binary search; the offsets never decrease)
-        uint64_t lo = 0, hi = seg.num_segments;
+        uint64_t lo = 0, hi = active ? seg.num_segments : 0;
         while (lo < hi) {
             const uint64_t mid = (lo + hi) >> 1;
             if (seg.start(mid) < row * kTileCols) lo = mid + 1;
             else hi = mid;
         }
         k0 = lo;
-        has_start = k0 < seg.num_segments && seg.start(k0) < n;
+        has_start = active && k0 < seg.num_segments && seg.start(k0) < n;
     } else {
-        k0 = (uint64_t(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-        if (k0 >= seg.num_segments) return;
-        const uint64_t p = seg.start(k0);
-        if (p >= n) return;                                         // empty segments at the very end
-        row = p / kTileCols;
-        if (k0 > 0 && seg.start(k0 - 1) / kTileCols == row) return;     // an earlier start of the row does it
-        if (row >= rows128) return;                                 // the incomplete last row: mode tail
+        k0 = (uint64_t(blockIdx.x) * blockDim.x + threadIdx.x) / kSegLanes;
+        active = k0 < seg.num_segments;
+        if (active) {
+            const uint64_t p = seg.start(k0);
+            row = p / kTileCols;
+            if (p >= n) active = false;                                          // empty segments at the very end
+            else if (k0 > 0 && seg.start(k0 - 1) / kTileCols == row) active = false;   // an earlier start of the row does it
+            else if (row >= rows128) active = false;                             // the incomplete last row: mode tail
+        }
+        has_start = active;
     }
     const uint64_t base = row * kTileCols;
-    const uint32_t count = uint32_t(n - base < kTileCols ? n - base : kTileCols);
-    // this lane's four elements and their start marks
-    uint32_t mark = 0;                     // bit i: a segment starts at column 4 * lane + i
+    const uint32_t count = !active ? 0u : uint32_t(n - base < kTileCols ? n - base : kTileCols);
+    // this lane's elements and their start marks
+    uint32_t mark = 0;                     // bit i: a segment starts at column kSegPerLane * sl + i
     uint32_t first_col = kTileCols, first_inner_col = kTileCols;    // first start of the row; first one that is not at column 0
     if (has_start) {
         for (uint64_t k = k0; k < seg.num_segments; ++k) {
             const uint64_t p = seg.start(k);
             if (p >= base + count) break;
             const uint32_t c = uint32_t(p - base);
-            if ((c >> 2) == uint32_t(lane)) mark |= 1u << (c & 3);
+            if (c / kSegPerLane == uint32_t(sl)) mark |= 1u << (c % kSegPerLane);
             if (first_col == kTileCols) first_col = c;
             if (c > 0 && first_inner_col == kTileCols) first_inner_col = c;
         }
     }
-    ValT x[4];
-    if (count == kTileCols) {              // a whole row: one aligned 4- or 8-byte load per lane
+    ValT x[kSegPerLane];
+#pragma unroll
+    for (int i = 0; i < kSegPerLane; ++i) x[i] = ValT(0);
+    if (count == kTileCols) {              // a whole row: aligned 16-byte loads
         if (IS_INT) {
-            const uint32_t w4 = reinterpret_cast<const uint32_t *>(reinterpret_cast<const int8_t *>(in) + base)[lane];
+            const uint4 w = reinterpret_cast<const uint4 *>(reinterpret_cast<const int8_t *>(in) + base)[sl];
+            const uint32_t wd[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) x[i] = ValT(int32_t(int8_t((w4 >> (8 * i)) & 0xFF)));
+            for (int i = 0; i < kSegPerLane; ++i) x[i] = ValT(int32_t(int8_t((wd[i >> 2] >> (8 * (i & 3))) & 0xFF)));
         } else {
-            const uint2 w8 = reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(in) + base)[lane];
-            const uint32_t h[4] = {w8.x & 0xFFFFu, w8.x >> 16, w8.y & 0xFFFFu, w8.y >> 16};
+            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint16_t *>(in) + base) + 2 * sl;
+            const uint4 wa = src[0], wb = src[1];
+            const uint32_t wd[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                x[i] = ValT((dtype == 2) ? __uint_as_float(h[i] << 16) : __half2float(__ushort_as_half(uint16_t(h[i]))));
+            for (int i = 0; i < kSegPerLane; ++i) {
+                const uint32_t h = (wd[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
+                x[i] = ValT((dtype == 2) ? __uint_as_float(h << 16) : __half2float(__ushort_as_half(uint16_t(h))));
+            }
         }
-    } else {
+    } else if (count > 0) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t c = 4 * lane + i;
-            x[i] = ValT(0);
+        for (int i = 0; i < kSegPerLane; ++i) {
+            const uint32_t c = kSegPerLane * sl + i;
             if (c < count) {
                 if (IS_INT) {
                     x[i] = ValT(int32_t(reinterpret_cast<const int8_t *>(in)[base + c]));
@@ -1617,12 +1632,12 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
             }
         }
     }
-    // scan with restarts: inside the lane, then across the lanes on (restarted?, value) pairs
-    ValT inc[4];
+    // scan with restarts: inside the lane, then across the lanes of the group on (restarted?, value) pairs
+    ValT inc[kSegPerLane];
     ValT run = ValT(0);
     bool cut = false;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kSegPerLane; ++i) {
         if (mark & (1u << i)) {
             run = ValT(0);
             cut = true;
@@ -1633,22 +1648,23 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
     ValT lane_val = run;
     bool lane_cut = cut;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const ValT v = __shfl_up_sync(0xffffffffu, lane_val, o);
-        const int f = __shfl_up_sync(0xffffffffu, int(lane_cut), o);
-        if (lane >= o) {
+    for (int o = 1; o < kSegLanes; o <<= 1) {
+        const ValT v = __shfl_up_sync(kFull, lane_val, o, kSegLanes);
+        const int f = __shfl_up_sync(kFull, int(lane_cut), o, kSegLanes);
+        if (sl >= o) {
             if (!lane_cut) lane_val += v;
             lane_cut = lane_cut || (f != 0);
         }
     }
-    ValT before = __shfl_up_sync(0xffffffffu, lane_val, 1);              // what the lanes to the left hand on
-    int before_cut = __shfl_up_sync(0xffffffffu, int(lane_cut), 1);
-    if (lane == 0) {
+    ValT before = __shfl_up_sync(kFull, lane_val, 1, kSegLanes);              // what the lanes to the left hand on
+    int before_cut = __shfl_up_sync(kFull, int(lane_cut), 1, kSegLanes);
+    if (sl == 0) {
         before = ValT(0);
         before_cut = 0;
     }
+    if (!active) return;                   // (no warp-wide operation below this line)
     if (MODE == kSegPrepare) {
-        if (lane == 31) {
+        if (sl == kSegLanes - 1) {
             rowflag[row] = uint8_t(kRowHasStart | (first_col == 0 ? kRowCutIn : 0));
             rowval[row] = IS_INT ? uint32_t(lane_val) : __float_as_uint(float(lane_val));
         }
@@ -1665,9 +1681,9 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
     const uint32_t from = (MODE == kSegTail) ? 0u : first_inner_col;
     bool open = !before_cut;               // still in the segment that entered the row (the carry applies)
     ValT left = before;                    // inclusive value of the element to the left, within its segment
-    uint32_t res[4];
+    uint32_t res[kSegPerLane];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kSegPerLane; ++i) {
         if (mark & (1u << i)) {
             open = false;
             left = ValT(0);
@@ -1681,15 +1697,18 @@ __global__ void __launch_bounds__(256) tcu_segment_rows_kernel(const void *in, v
         res[i] = bits;
         left = incl;
     }
-    // write: one 16-byte store when all four of the lane's elements are to be written, else element by element
-    uint32_t *const o32 = reinterpret_cast<uint32_t *>(out) + base + 4 * lane;
-    const uint32_t c0 = 4 * lane;
-    if ((MODE == kSegTail || c0 >= from) && c0 + 3 < count) {
-        *reinterpret_cast<uint4 *>(o32) = make_uint4(res[0], res[1], res[2], res[3]);
-    } else {
+    // write: 16-byte stores for every four elements that are all to be written, else element by element
+    uint32_t *const o32 = reinterpret_cast<uint32_t *>(out) + base + kSegPerLane * sl;
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if ((MODE == kSegTail || c0 + i >= from) && c0 + i < count) o32[i] = res[i];
+    for (int q = 0; q < kSegPerLane / 4; ++q) {
+        const uint32_t c0 = kSegPerLane * sl + 4 * q;
+        if ((MODE == kSegTail || c0 >= from) && c0 + 3 < count) {
+            *reinterpret_cast<uint4 *>(o32 + 4 * q) = make_uint4(res[4 * q], res[4 * q + 1], res[4 * q + 2], res[4 * q + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if ((MODE == kSegTail || c0 + i >= from) && c0 + i < count) o32[4 * q + i] = res[4 * q + i];
+        }
     }
 }
 
