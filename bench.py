@@ -587,6 +587,11 @@ def run_ours(args):
                 # the same scans in the two-sweep structure (reduce, scan the totals, scan with every carry known)
                 extra["C3_two_sweep"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, variant=1)[0])
                 extra["f16_n2p28_two_sweep"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, variant=1)[0])
+                # ... with the scan of the tile totals sent through the tensor-core scan again (narrow terms, one inner scan each)
+                extra["C3_two_sweep_totals_by_scan"] = frac(time_extra(B, torch, d_in, 1, n, 0, 16, ws_ptr, ws_bytes, variant=1,
+                                                                       upper_level_path=1)[0])
+                extra["f16_n2p28_two_sweep_totals_by_scan"] = frac(time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes,
+                                                                              variant=1, upper_level_path=1)[0])
                 # upper level (scan over the 128 row totals) as a tcgen05 product on exact narrow terms
                 # (path 2: the chunk level inside a row as a product as well)
                 for path in (1, 2):

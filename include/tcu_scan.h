@@ -104,7 +104,14 @@ typedef struct {
                                        upper triangular ones matrix, instead of a chain of additions along
                                        the row (for s = 128 a row is one chunk and 2 means 1).
                                    Integer results are identical, floating-point results satisfy the
-                                   same tolerance.  The level across tiles stays a look-back on CUDA cores. */
+                                   same tolerance.  In the single-pass variant the level across tiles stays a
+                                   look-back on CUDA cores; in the two-sweep variant (variant = 1) a value >= 1
+                                   also sends the scan of the tile totals (Section 2.2 step 3) through the
+                                   tensor-core scan: each total is split exactly into narrow terms (four signed
+                                   base-256 digits; the fp32-rounded total in three bf16 terms), every term
+                                   array is scanned by an inner call of this library with the same s and the
+                                   same value of this option, and the scanned terms are recombined (shifts
+                                   and adds mod 2^32; three fp32 sums added in fp64). */
     uint32_t down_sweep_path;   /* Paper Section 2, matrix B_s, and the discussion's remark that the tensor
                                    unit is used at O(1/s) in the down-sweep.  1 = fp16 / bf16 scans with
                                    s = 128 add each row's carry to the whole row by a tcgen05 product
@@ -129,8 +136,11 @@ typedef struct {
  * (rows = 1 for the single-array calls).  Holds the per-tile {flag, aggregate / inclusive
  * prefix} records of the cross-tile carry scan (Section 2.2 steps 2-3: segment totals and
  * their scan); when cols is not a multiple of 16 and rows > 1, also the per-row boundary
- * notes of the segmented path.  Never fails; returns a small non-zero size even for empty
- * problems. */
+ * notes of the segmented path; for a single array, also the scratch of the two-sweep variant
+ * when it scans the tile totals with the library's own scan (tcu_scan_options_t: variant = 1
+ * with upper_level_path >= 1) - the size covers every option of tcu_scan_ex, about 40 bytes
+ * per 128 x 128-element tile in all.  Never fails; returns a small non-zero size even for
+ * empty problems. */
 size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s);
 
 /* Clear a workspace (asynchronous memset on `stream`).  Must run once before the first

@@ -131,6 +131,7 @@ struct Call {
     tcu_dtype_t dt = TCU_I8_I32;
     int s = 16;
     bool exclusive = false, level0 = false, two_sweep = false;
+    bool nested = false;                 // an inner scan over the narrow terms of the tile totals (two-sweep variant)
     int upper_path = 0, down_path = 0, max_ctas = 0;
     const void *d_carry_in = nullptr;
     void *d_carry_out = nullptr;
@@ -155,8 +156,19 @@ size_t seg_flag_offset(uint64_t n) { return round_up(record_bytes(tiles_for(1, n
 size_t seg_rows(uint64_t n) { return size_t(tiles_for(1, n)) * kTileRows + 1; }
 size_t seg_val_offset(uint64_t n) { return seg_flag_offset(n) + round_up(seg_rows(n), 256); }
 size_t seg_workspace_bytes(uint64_t n) { return seg_val_offset(n) + round_up(4 * seg_rows(n), 256); }
+// Two-sweep variant with the scan of the tile totals done by this library's own scan (one array per narrow term of
+// the totals): behind the records lie the term arrays (at most 4 planes of T one- or two-byte terms), their scans
+// (4 planes of T four-byte sums) and the workspace of those inner scans.
+size_t nested_offset(uint64_t tiles) { return round_up(record_bytes(tiles), 256); }
+size_t nested_in_stride(uint64_t tiles) { return round_up(2 * size_t(tiles), 256); }
+size_t nested_out_stride(uint64_t tiles) { return round_up(4 * size_t(tiles), 256); }
+size_t nested_ws_bytes(uint64_t tiles) { return round_up(record_bytes(tiles_for(1, tiles)), 256); }
+size_t nested_bytes(uint64_t tiles) { return 4 * nested_in_stride(tiles) + 4 * nested_out_stride(tiles) + nested_ws_bytes(tiles); }
+bool totals_by_scan(const Call &c);
 size_t needed_workspace(const Call &c) {
-    return c.segmented ? seg_workspace_bytes(uint64_t(c.rows) * c.cols) : record_bytes(tiles_for(c.rows, c.cols));
+    if (c.segmented) return seg_workspace_bytes(uint64_t(c.rows) * c.cols);
+    const uint64_t tiles = tiles_for(c.rows, c.cols);
+    return totals_by_scan(c) ? nested_offset(tiles) + nested_bytes(tiles) : record_bytes(tiles);
 }
 
 // Host-side checks of a call; nothing has been queued on the stream when this returns an error.
@@ -188,6 +200,42 @@ tcu_status_t check_call(const Call &c) {
     if (tiles >= (1ull << 31)) return TCU_ERR_UNSUPPORTED;
     if (c.max_ctas < 0 || c.upper_path < 0 || c.upper_path > 2 || c.down_path < 0 || c.down_path > 1) return TCU_ERR_INVALID_ARG;
     return TCU_OK;
+}
+
+bool totals_by_scan(const Call &c) { return c.two_sweep && c.upper_path >= 1 && !c.nested; }
+
+tcu_status_t scan_impl(const Call &c);
+Call make_call(const void *d_in, void *d_out, size_t rows, size_t cols, tcu_dtype_t dt, int s, bool exclusive, void *d_ws,
+               size_t ws_bytes, cudaStream_t stream);
+
+// Sweep 1.5 of the two-sweep variant when the upper levels are asked for as products: the tile totals (already in the
+// records) are split into narrow terms, every term array is scanned by an ordinary call of this library, and the
+// scanned terms are recombined into the inclusive records that sweep 2 expects.
+tcu_status_t scan_totals_by_scan(const Call &c, uint64_t tiles, uint64_t *inner_mma) {
+    uint8_t *base = reinterpret_cast<uint8_t *>(c.d_ws) + nested_offset(tiles);
+    const bool is_int = c.dt == TCU_I8_I32;
+    const int terms = is_int ? kSplitTermsInt : kSplitTermsFloat;
+    const size_t in_stride = nested_in_stride(tiles), out_stride = nested_out_stride(tiles);
+    uint8_t *planes = base, *sums = base + 4 * in_stride, *inner_ws = sums + 4 * out_stride;
+    const unsigned blocks = unsigned((tiles + 255) / 256);
+    if (is_int) tcu_totals_split_kernel<true><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), planes, uint32_t(in_stride));
+    else tcu_totals_split_kernel<false><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), planes, uint32_t(in_stride));
+    if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+    for (int b = 0; b < terms; ++b) {
+        Call in = make_call(planes + size_t(b) * in_stride, sums + size_t(b) * out_stride, 1, size_t(tiles),
+                            is_int ? TCU_I8_I32 : TCU_BF16_F32, c.s, false, inner_ws, nested_ws_bytes(tiles), c.stream);
+        in.nested = true;
+        in.upper_path = c.upper_path;            // the inner scans take the same optional product levels
+        in.spin_limit = c.spin_limit;
+        tcu_scan_stats_t inner;
+        in.stats_out = &inner;
+        const tcu_status_t st = scan_impl(in);
+        if (st != TCU_OK) return st;
+        *inner_mma += inner.mma_instructions;
+    }
+    if (is_int) tcu_totals_combine_kernel<true><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), sums, uint32_t(out_stride));
+    else tcu_totals_combine_kernel<false><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), sums, uint32_t(out_stride));
+    return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
 }
 
 tcu_status_t scan_impl(const Call &c) {
@@ -315,14 +363,20 @@ tcu_status_t scan_impl(const Call &c) {
         if (two_sweep) {
             // sweep 1: one total per tile; then their scan, written as the records sweep 2 looks back over
             const uint64_t valid = uint64_t(rows128) * kTileCols;
-            if (dt == TCU_I8_I32) {
-                tcu_tile_totals_kernel<true><<<unsigned(tiles), 256, 0, stream>>>(d_in, d_ws, valid, dt);
-                tcu_totals_scan_kernel<true><<<1, 1024, 0, stream>>>(d_ws, uint32_t(tiles));
-            } else {
-                tcu_tile_totals_kernel<false><<<unsigned(tiles), 256, 0, stream>>>(d_in, d_ws, valid, dt);
-                tcu_totals_scan_kernel<false><<<1, 1024, 0, stream>>>(d_ws, uint32_t(tiles));
-            }
+            if (dt == TCU_I8_I32) tcu_tile_totals_kernel<true><<<unsigned(tiles), 256, 0, stream>>>(d_in, d_ws, valid, dt);
+            else tcu_tile_totals_kernel<false><<<unsigned(tiles), 256, 0, stream>>>(d_in, d_ws, valid, dt);
             if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+            if (totals_by_scan(c)) {
+                uint64_t inner_mma = 0;
+                const tcu_status_t ts = scan_totals_by_scan(c, tiles, &inner_mma);
+                if (ts != TCU_OK) return ts;
+                st.mma_instructions += inner_mma;
+                st.levels_used += 1;             // (the totals go through a scan of their own)
+            } else {
+                if (dt == TCU_I8_I32) tcu_totals_scan_kernel<true><<<1, 1024, 0, stream>>>(d_ws, uint32_t(tiles));
+                else tcu_totals_scan_kernel<false><<<1, 1024, 0, stream>>>(d_ws, uint32_t(tiles));
+                if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+            }
         }
         dim3 grid(unsigned(tiles < ctas ? tiles : ctas));
         st.grid = grid.x;
@@ -451,7 +505,9 @@ size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s)
     (void)dt;
     (void)s;
     if (rows > 1 && cols % 16 != 0) return seg_workspace_bytes(uint64_t(rows) * cols);   // rows become segments of one array
-    return record_bytes(tiles_for(rows, cols));
+    const uint64_t tiles = tiles_for(rows, cols);
+    // (room for every option: the two-sweep variant with the totals scanned by this library's own scan needs the most)
+    return rows > 1 ? record_bytes(tiles) : nested_offset(tiles) + nested_bytes(tiles);
 }
 
 tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t stream) {

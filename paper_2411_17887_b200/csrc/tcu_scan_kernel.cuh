@@ -1526,6 +1526,68 @@ __global__ void __launch_bounds__(1024) tcu_totals_scan_kernel(void *ws, uint32_
     }
 }
 
+// ---- two-sweep variant with the scan of the tile totals done by the tensor-core scan itself (Section 2.2 step 3: the
+// totals of the segments are scanned with Algorithm 1 again).  Tile totals are 32-bit integers or doubles, not
+// tensor-core input types, so each is first split exactly into narrow terms, every term forms an array of its own that
+// goes through the ordinary scan of this library, and the scanned terms are recombined:
+//   integer: four signed base-256 digits d0..d3 with d0 + 256 d1 + 65536 d2 + 16777216 d3 = total (mod 2^32); the scans
+//            are exact mod 2^32, so is the recombination sum_b (scan_b << 8 b);
+//   float:   the total rounded to fp32 and cut into three bf16 terms hi + mid + lo (8 significant bits each, exact);
+//            the three fp32 scans are added in fp64.
+constexpr int kSplitTermsInt = 4, kSplitTermsFloat = 3;
+template <bool IS_INT>
+__global__ void __launch_bounds__(256) tcu_totals_split_kernel(const void *ws, uint32_t tiles, uint8_t *planes, uint32_t plane_stride) {
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= tiles) return;
+    const uint64_t *rec = reinterpret_cast<const uint64_t *>(reinterpret_cast<const uint8_t *>(ws) + kHeaderBytes);
+    const uint64_t bits = rec[2 * size_t(t) + 1];
+    if (IS_INT) {
+        uint32_t v = uint32_t(bits);
+#pragma unroll
+        for (int b = 0; b < kSplitTermsInt; ++b) {
+            const int32_t d = int32_t(int8_t(v & 0xFFu));             // digit in [-128, 127]
+            reinterpret_cast<int8_t *>(planes + size_t(b) * plane_stride)[t] = int8_t(d);
+            v = (v - uint32_t(d)) >> 8;                                // exact: the low byte is zero now
+        }
+    } else {
+        const float f = float(__longlong_as_double((long long)bits));
+        const uint32_t hi = __float_as_uint(f) & 0xFFFF0000u;
+        const float r1 = f - __uint_as_float(hi);
+        const uint32_t mid = __float_as_uint(r1) & 0xFFFF0000u;
+        const float r2 = r1 - __uint_as_float(mid);
+        const uint32_t lo = __float_as_uint(r2) & 0xFFFF0000u;          // r2 has at most 8 significant bits
+        reinterpret_cast<uint16_t *>(planes + 0 * size_t(plane_stride))[t] = uint16_t(hi >> 16);
+        reinterpret_cast<uint16_t *>(planes + 1 * size_t(plane_stride))[t] = uint16_t(mid >> 16);
+        reinterpret_cast<uint16_t *>(planes + 2 * size_t(plane_stride))[t] = uint16_t(lo >> 16);
+    }
+}
+
+// Recombines the scanned terms into the records sweep 2 looks back over: {INCLUSIVE, sum of the totals of tiles 0..t}.
+template <bool IS_INT>
+__global__ void __launch_bounds__(256) tcu_totals_combine_kernel(void *ws, uint32_t tiles, const uint8_t *sums, uint32_t sum_stride) {
+    using CO = CarryOps<IS_INT>;
+    using CarryT = typename CO::T;
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= tiles) return;
+    const WsHeader *hdr = reinterpret_cast<const WsHeader *>(ws);
+    uint64_t *rec = reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(ws) + kHeaderBytes);
+    const uint64_t flag = (uint64_t(hdr->epoch + 1) << 2) | kStatusInclusive;   // the epoch the main kernel will use
+    CarryT prefix = CarryT(0);
+    if (IS_INT) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int b = 0; b < kSplitTermsInt; ++b) acc += reinterpret_cast<const uint32_t *>(sums + size_t(b) * sum_stride)[t] << (8 * b);
+        prefix = CarryT(acc);
+    } else {
+        double acc = 0.0;
+#pragma unroll
+        for (int b = 0; b < kSplitTermsFloat; ++b) acc += double(reinterpret_cast<const float *>(sums + size_t(b) * sum_stride)[t]);
+        prefix = CarryT(acc);
+    }
+    rec[2 * size_t(t) + 1] = CO::enc(prefix);
+    rec[2 * size_t(t)] = flag;
+}
+
 // ---- segmented scan (Section 2.2 with caller-given segments): the rows that hold a segment start ---------------
 // The array is cut into rows of 128 elements, counted from its start.  A row in which no segment starts belongs to
 // one segment and goes through the tensor-core path unchanged.  A row that holds starts is summarised for that path

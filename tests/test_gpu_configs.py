@@ -89,6 +89,19 @@ def test_beyond_four_gigabytes_of_output():
     compare_piecewise(got, x, "i8", True)
 
 
+def test_two_sweep_with_scanned_totals_beyond_one_inner_tile():
+    # more than 128 x 128 tile totals: the inner scans over the terms of the totals have tiles and a tail of their own
+    from tests.gpu_util import Runner
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    n = (16384 + 300) * 16384 + 5
+    x = inputs.int8_uniform(n, -127, 127, 41)
+    big = Runner(1, n)
+    got = big.run(x, "i8", 16, variant=1, upper_level_path=1)
+    compare_piecewise(got, x, "i8", False)
+    assert big.stats["variant"] == 1 and big.stats["upper_level_path"] == 1 and big.stats["tiles"] == 16384 + 300
+
+
 def test_segmented_at_the_headline_size():
     # n = 2^28 int8 cut at random points (mean segment 2^12, some empty segments), in the launch configuration the
     # benchmark times; every output compared with the oracle's per-segment loop

@@ -164,6 +164,38 @@ def test_two_sweep_variant_matches_oracle(runner, dtype):
     check(runner, gen(dtype, 5 * TILE + 3, 17), dtype, 16)
 
 
+@pytest.mark.parametrize("dtype", ["i8", "f16", "bf16"])
+def test_two_sweep_with_the_totals_scanned_by_the_library_itself(runner, dtype):
+    # Section 2.2 step 3 literally: the tile totals, split into exact narrow terms, go through the tensor-core scan again
+    # (one inner scan per term) and are recombined; integers stay bit-exact, floats within the tolerance
+    from tests.gpu_util import check
+    cases = [(TILE, 16, 1), (37 * TILE + 128 * 5 + 9, 64, 1), (128 * TILE, 16, 2), (1500 * TILE + 77, 16, 1),
+             (1500 * TILE + 77, 128, 2), (130 * TILE + 1, 64, 2)]
+    for n, s, path in cases:
+        for exclusive in (False, True):
+            check(runner, gen(dtype, n, 5000 + n % 907), dtype, s, exclusive, variant=1, upper_level_path=path)
+            st = runner.stats
+            assert st["variant"] == 1 and st["upper_level_path"] == path
+    if dtype == "i8":
+        # tile totals of +-2 080 768 (digits of both signs, carries between the digits), prefix sums that wrap twice
+        for value in (127, -127, -128):
+            x = np.full(1 << 26, value, dtype=np.int8)
+            check(runner, x, "i8", 16, variant=1, upper_level_path=1)
+    else:
+        # all-ones input: every total and every prefix is an integer below 2^24, so the result must be exact
+        n = 900 * TILE + 128 * 3 + 5
+        got = runner.run(inputs_ones(dtype, n), dtype, 16, variant=1, upper_level_path=1)
+        assert np.array_equal(got, np.arange(1, n + 1, dtype=np.float32))
+    # the single-pass path still works on the same workspace afterwards
+    check(runner, gen(dtype, 5 * TILE + 3, 17), dtype, 16)
+
+
+def inputs_ones(dtype, n):
+    if dtype == "f16":
+        return np.ones(n, dtype=np.float16)
+    return np.full(n, 0x3F80, dtype=np.uint16)          # bf16 1.0
+
+
 def test_result_does_not_depend_on_the_number_of_ctas(runner):
     # the p of the paper's p-TCU bound: any number of persistent CTAs gives the same integers
     from paper_2411_17887_b200 import binding as B

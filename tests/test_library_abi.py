@@ -51,10 +51,16 @@ def test_workspace_bytes(B):
     tile = 128 * 128
     base = B.tcu_scan_workspace_bytes(1, 0, 0, 16)
     assert base >= 256
-    assert B.tcu_scan_workspace_bytes(1, tile, 0, 16) == base + 16
-    assert B.tcu_scan_workspace_bytes(1, tile + 128, 1, 64) == base + 32
-    assert B.tcu_scan_workspace_bytes(1, 1 << 28, 0, 16) == base + 16 * (1 << 14)
-    assert B.tcu_scan_workspace_bytes(4096, 65536, 2, 16) == base + 16 * 4096 * 4
+    # single arrays: 16 bytes of record per tile, plus room for the two-sweep variant's scan of the tile totals by the
+    # library itself (four term arrays, their four scans, the inner scans' own records): a few dozen bytes per tile
+    one = B.tcu_scan_workspace_bytes(1, tile, 0, 16)
+    assert base < one <= base + 4096
+    assert one <= B.tcu_scan_workspace_bytes(1, tile + 128, 1, 64) <= one + 4096
+    big = B.tcu_scan_workspace_bytes(1, 1 << 28, 0, 16)
+    assert 16 * (1 << 14) < big <= 48 * (1 << 14)
+    assert big % 256 == 0 and one % 256 == 0
+    # dense rows: records only
+    assert B.tcu_scan_workspace_bytes(4096, 65536, 2, 16) == 256 + 16 + 16 * 4096 * 4
 
 
 def test_argument_checks_return_before_any_launch(B):
