@@ -596,7 +596,10 @@ tcu_status_t tcu_scan_inclusive_noalloc(const void *d_in, void *d_out, size_t n,
     if (st != TCU_OK) return st;
     // The scratch still holds the records of whatever call used it last.  Everything the kernels
     // expect to find at zero (header counters, the records of this call's tiles) is cleared here.
-    const size_t used = tcu_scan_workspace_bytes(1, n, dt, s);
+    const size_t used = record_bytes(tiles_for(1, n));           // (never more than the array: n was checked above)
+    static_assert(kNoAllocScratchBytes >= size_t(kHeaderBytes) + 16 * (size_t(TCU_SCAN_NOALLOC_MAX_ELEMENTS) / kTileElems) + 16,
+                  "the built-in scratch holds the records of the largest scan it accepts");
+    if (used > kNoAllocScratchBytes) return TCU_ERR_TOO_LARGE;
     if (cudaMemsetAsync(scratch, 0, used, stream) != cudaSuccess) return TCU_ERR_CUDA;
     c.d_ws = scratch;
     return scan_impl(c);

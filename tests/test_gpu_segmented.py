@@ -138,7 +138,8 @@ def test_segmented_argument_checks():
     o = torch.zeros(1024, dtype=torch.int32, device="cuda")
     off = torch.tensor([0, 1024], dtype=torch.int64, device="cuda")
     ws_bytes = B.tcu_scan_segmented_workspace_bytes(1024, 0, 16)
-    assert ws_bytes > B.tcu_scan_workspace_bytes(1, 1024, 0, 16)
+    # beside the tile records: one flag byte and one 4-byte value per row of 128 elements
+    assert B.tcu_scan_segmented_workspace_bytes(1 << 24, 0, 16) >= 256 + 5 * ((1 << 24) // 128) + 16 * ((1 << 24) // TILE)
     ws = torch.zeros(ws_bytes + 256, dtype=torch.uint8, device="cuda")
     ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
     assert B.tcu_scan_segmented(d, o, 1024, None, 1, 0, 16, 0, ptr, ws_bytes, 0) == B.TCU_ERR_INVALID_ARG
