@@ -4,6 +4,7 @@
     python bench.py --gpus N --steps K --warmup W            # this library (CUDA, through the C ABI)
     python bench.py --impl reference --steps K --warmup W    # the CPU oracle on the host cores
     python bench.py --fixed-cost                             # where the microseconds of a small launch go
+    python bench.py --wait-counters | --tile-trace           # debug build: waits per role; the life of a tile
     python bench.py --profile ...                            # the bare loop that is wrapped in ncu
 
 A step is one scan of the headline workload: n = 2^28 int8 values uniform in [-127, 127],
@@ -355,6 +356,69 @@ def wait_counters(args):
     print(json.dumps({"wait_counters": report, "sm_ghz_assumed": ghz}))
 
 
+def tile_trace(args):
+    """The life of a tile and the rate at which tiles are completed over a launch: loads the debug build of the
+    library (-DTCU_PROFILE), attaches a buffer of eight time stamps per tile (claimed, row-total product issued, totals
+    warps woken, total published, walk started, carry known, store started, stored; ``%globaltimer``), runs one scan
+    per workload and prints (a) the median time from the claim to each point for tiles of the first waves and of the
+    steady state, (b) the algorithmic GB/s at which tiles are stored between given fractions of the launch.  The
+    stamps slow the kernel by a few per cent; the point is where the time goes, and whether the middle of a launch runs
+    at the rate of a plain copy of the same traffic."""
+    import ctypes
+    import numpy as np
+    import torch
+    from paper_2411_17887_b200 import build as lib_build
+    lib = ctypes.CDLL(lib_build.build_profile())
+    vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    lib.tcu_scan_workspace_bytes.argtypes = [sz, sz, ci, ci]
+    lib.tcu_scan_workspace_bytes.restype = sz
+    lib.tcu_scan_workspace_init.argtypes = [vp, sz, vp]
+    lib.tcu_scan_inclusive.argtypes = [vp, vp, sz, ci, ci, vp, sz, vp]
+    lib.tcu_scan_debug_set_trace_buffer.argtypes = [vp]
+    torch.cuda.set_device(0)
+    st = torch.cuda.current_stream().cuda_stream
+    g = torch.Generator(device="cuda").manual_seed(1)
+    points = ["claimed", "row_total_product_issued", "totals_warps_woken", "total_published", "walk_started", "carry_known",
+              "store_started", "stored"]
+    report = []
+    for label, logn, dt in [("C3 int8 n=2^28", 28, 0), ("fp16 n=2^28", 28, 1), ("C5 fp16 n=2^26", 26, 1)]:
+        n = 1 << logn
+        tiles = n // (128 * 128)
+        ws_bytes = lib.tcu_scan_workspace_bytes(1, n, dt, 16)
+        ws = torch.zeros(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+        ws_ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+        x = (torch.randint(-127, 128, (n,), device="cuda", dtype=torch.int8, generator=g) if dt == 0
+             else (torch.rand(n, device="cuda", generator=g) * 2 - 1).half())
+        out = torch.empty(n, dtype=torch.int32, device="cuda")
+        trace = torch.zeros(tiles * 8, dtype=torch.int64, device="cuda")
+        lib.tcu_scan_debug_set_trace_buffer(None)
+        for _ in range(3):
+            assert lib.tcu_scan_inclusive(x.data_ptr(), out.data_ptr(), n, dt, 16, ws_ptr, ws_bytes, st) == 0
+        torch.cuda.synchronize()
+        assert lib.tcu_scan_debug_set_trace_buffer(trace.data_ptr()) == 0
+        assert lib.tcu_scan_inclusive(x.data_ptr(), out.data_ptr(), n, dt, 16, ws_ptr, ws_bytes, st) == 0
+        torch.cuda.synchronize()
+        lib.tcu_scan_debug_set_trace_buffer(None)
+        T = trace.cpu().numpy().reshape(tiles, 8).astype(np.int64)
+        t0 = int(T[:, 0].min())
+        entry = {"workload": label, "tiles": tiles, "us_since_claim_median": {}, "stored_rate_GBps": {}}
+        for lo, hi in [(0, 32), (32, 148), (148, 740), (740, 1480), (tiles // 2, tiles // 2 + 1000), (tiles - 1000, tiles - 300)]:
+            med = np.median((T[lo:hi] - T[lo:hi, :1]) / 1e3, axis=0)
+            entry["us_since_claim_median"][f"tiles {lo}-{hi}"] = {nm: round(float(v), 2) for nm, v in zip(points, med)}
+        stored = np.sort((T[:, 7] - t0) / 1e3)
+        claimed = np.sort((T[:, 0] - t0) / 1e3)
+        bpe = 5 if dt == 0 else 6
+        entry["us_after_first_claim"] = {"first_stored": round(float(stored[0]), 1), "last_claimed": round(float(claimed[-1]), 1),
+                                         "99pct_stored": round(float(stored[-tiles // 100]), 1), "last_stored": round(float(stored[-1]), 1)}
+        for a, b in [(0.0, 0.05), (0.05, 0.95), (0.1, 0.5), (0.5, 0.9), (0.95, 1.0)]:
+            ia, ib = int(a * tiles), min(int(b * tiles), tiles - 1)
+            entry["stored_rate_GBps"][f"{a:.2f}-{b:.2f}"] = round((ib - ia) * 128 * 128 * bpe / (stored[ib] - stored[ia]) / 1e3)
+        entry["whole_launch_GBps"] = round(n * bpe / float(stored[-1]) / 1e3)
+        report.append(entry)
+        del x, out, trace, ws
+    print(json.dumps({"tile_trace": report}))
+
+
 def run_sharded(args):
     """One array of 2^n_log2 int8 elements split into contiguous shards, one per rank (strong scaling): every step
     each rank takes the total of its shard, the totals are all-gathered (8 bytes per rank), each rank sums the totals
@@ -677,6 +741,8 @@ def main():
                     help="one array split over the ranks (strong scaling) instead of one array per rank")
     ap.add_argument("--wait-counters", action="store_true",
                     help="debug build of the library: where each role of the kernel waits, at the headline size")
+    ap.add_argument("--tile-trace", action="store_true",
+                    help="debug build: eight time stamps per tile; the life of a tile and the completion rate over a launch")
     ap.add_argument("--fixed-cost", action="store_true",
                     help="break the time of small launches (C1, C2, C5) into phases with the kernel's time stamps")
     args = ap.parse_args()
@@ -686,6 +752,8 @@ def main():
         fixed_cost(args)
     elif args.wait_counters:
         wait_counters(args)
+    elif args.tile_trace:
+        tile_trace(args)
     elif args.sharded:
         run_sharded(args)
     else:
