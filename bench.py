@@ -631,6 +631,20 @@ def run_ours(args):
                 extra["C4_4096x65536_bf16"] = frac(time_extra(B, torch, xb, 4096, 65536, 2, 16, ws_ptr, ws_bytes)[0])
                 del xb
                 extra["C1_n2p16_i8"] = time_extra(B, torch, d_in, 1, 1 << 16, 0, 16, ws_ptr, ws_bytes, reps=200)[0]
+                # the same 64 Ki-element scan replayed from a CUDA graph of 20 launches: the host's 3-6 us per call
+                # (ctypes, tensor-map encoding, launch) are out of the loop
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph):
+                    cap = torch.cuda.current_stream().cuda_stream
+                    for _ in range(20):
+                        B.check(B.tcu_scan_inclusive(d_in, d_out, 1 << 16, 0, 16, ws_ptr, ws_bytes, cap))
+                for _ in range(3):
+                    graph.replay()
+                torch.cuda.synchronize()
+                ms_g = Timer(torch).loop(graph.replay, 25) / 20
+                extra["C1_n2p16_i8_cuda_graph"] = {"us": round(1e3 * ms_g, 2), "GBps": round(5 * (1 << 16) / (ms_g * 1e-3) / 1e9, 1)}
+                B.check(B.tcu_scan_device_status(ws_ptr, stream))
+                del graph
                 # plain widening copies with the scans' read / write mixes (1 : 4 and 2 : 4), no dependence between
                 # elements: what the memory system gives that mix when nothing has to be carried along
                 d_out_f = d_out.view(torch.float32)
