@@ -679,6 +679,9 @@ def run_ours(args):
                 for path in (0, 1):
                     extra[f"f16_n2p28_s128_down_sweep_path{path}"] = frac(
                         time_extra(B, torch, xf, 1, 1 << 28, 1, 128, ws_ptr, ws_bytes, down_sweep_path=path)[0])
+                # the same for s = 16: one carry per chunk, from the chunk-level product (upper_level_path = 2)
+                extra["f16_n2p28_s16_upper_level_path2_down_sweep_path1"] = frac(
+                    time_extra(B, torch, xf, 1, 1 << 28, 1, 16, ws_ptr, ws_bytes, upper_level_path=2, down_sweep_path=1)[0])
                 del xf
                 # segmented scan of the headline array: random cut points, mean segment length 2^10, 2^14, 2^18
                 for logm in (10, 14, 18):

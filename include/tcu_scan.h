@@ -113,10 +113,15 @@ typedef struct {
                                    same value of this option, and the scanned terms are recombined (shifts
                                    and adds mod 2^32; three fp32 sums added in fp64). */
     uint32_t down_sweep_path;   /* Paper Section 2, matrix B_s, and the discussion's remark that the tensor
-                                   unit is used at O(1/s) in the down-sweep.  1 = fp16 / bf16 scans with
-                                   s = 128 add each row's carry to the whole row by a tcgen05 product
-                                   (accumulator += C * ones, C holding the carry split exactly into three
-                                   bf16 terms) instead of one vector add per element; ignored otherwise. */
+                                   unit is used at O(1/s) in the down-sweep.  1 = fp16 / bf16 scans add the
+                                   carries by a tcgen05 product instead of one vector add per element:
+                                   with s = 128, each row's carry to the whole row (accumulator += C * ones,
+                                   C holding the carry split exactly into three bf16 terms); with s < 128
+                                   and upper_level_path = 2 (which provides the carries of the chunks), each
+                                   chunk's carry to the s elements of the chunk (accumulator += C * E, C
+                                   holding the 128 / s carries of a row in three bf16 terms each, E a 0 / 1
+                                   matrix that selects the chunk of every column).  Ignored otherwise
+                                   (integer scans: no pair of 8-bit operands adds a 32-bit carry). */
     uint32_t max_ctas;          /* 0 = one persistent CTA per SM; otherwise at most this many.  One CTA owns
                                    one SM's tensor core, so this is the p of the paper's p-TCU time bound
                                    O(n(1 + l/s^2)/p + (s^2 + l) log_s n) (Section 2.2, last paragraph).

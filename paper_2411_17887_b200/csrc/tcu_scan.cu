@@ -262,9 +262,12 @@ tcu_status_t scan_impl(const Call &c) {
     const uint32_t stage_bytes = kTileElems * eb;
     const bool upper_tc = c.upper_path >= 1 && !c.segmented && !level0;
     const bool chunk_tc = c.upper_path == 2 && s < kTileCols && !c.segmented && !level0;
-    const bool down_tc = (dt != TCU_I8_I32) && s == 128 && !level0 && c.down_path == 1 && !c.segmented;
+    // the carry add as a product: for s = 128 one carry per row; for s < 128 one per chunk, which needs the chunk totals
+    // out of the accumulator first, i.e. the chunk-product variant (upper_level_path = 2)
+    const bool chunk_down = chunk_tc && (dt != TCU_I8_I32) && c.down_path == 1;
+    const bool down_tc = ((dt != TCU_I8_I32) && s == 128 && !level0 && c.down_path == 1 && !c.segmented) || chunk_down;
     const size_t fixed = kConstOffset + kOnesBytes + b_bytes + size_t(kOutRingBytes) + (upper_tc ? (dt == TCU_I8_I32 ? kUpperBytesInt : kUpperBytesFloat) : 0) +
-                         (down_tc ? kDownBytes : 0) + (chunk_tc ? kChunkBytes : 0) + (c.segmented ? kSegRingBytes : 0) + 1024;  // + alignment slack
+                         (down_tc && !chunk_down ? kDownBytes : 0) + (chunk_tc ? kChunkBytes : 0) + (chunk_down ? kAtomBytes : 0) + (c.segmented ? kSegRingBytes : 0) + 1024;  // + alignment slack
     int in_stages = int((232448 - fixed) / stage_bytes);
     if (in_stages > kUseInStages) in_stages = kUseInStages;
     if (in_stages < 2) return TCU_ERR_UNSUPPORTED;
@@ -281,7 +284,7 @@ tcu_status_t scan_impl(const Call &c) {
     st.upper_level_path = upper_tc ? uint32_t(c.upper_path) : 0;
     st.down_sweep_path = down_tc ? 1 : 0;
     st.tiles = tiles;
-    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? (dt == TCU_I8_I32 ? 4 : 8) : 0) + (chunk_tc ? (dt == TCU_I8_I32 ? 1 : 2) : 0) + (down_tc ? 1 : 0));  // U_s products + row-total products
+    st.mma_instructions = tiles * uint64_t((kTileCols / seff) * (seff / per32) + kTileCols / per32 + (upper_tc ? (dt == TCU_I8_I32 ? 4 : 8) : 0) + (chunk_tc ? (dt == TCU_I8_I32 ? 1 : 2) : 0) + (chunk_down ? (3 * (kTileCols / s) + 15) / 16 : (down_tc ? 1 : 0)));  // U_s products + row-total products
     st.sxs_products = tiles * uint64_t(kTileElems / (s * s));
     // product level, chain over the chunks of a row (absent when s = 128), scan over the 128 rows,
     // scan over the tiles (absent for a single tile), carry add

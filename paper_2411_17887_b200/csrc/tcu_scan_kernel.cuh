@@ -463,6 +463,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     uint8_t *down_b = down_a + kStoreGroups * kAtomBytes;
     uint8_t *chunk_a = upper_a + (use_upper ? (IS_INT ? kUpperBytesInt : kUpperBytesFloat) : 0);   // only present in the CHUNK_TC variant
     uint8_t *chunk_b = chunk_a + kStoreGroups * kAtomBytes;
+    uint8_t *chunk_sel = chunk_b + kChunkConstBytes;       // only present in the CHUNK_TC variant with use_down
 
     WsHeader *hdr = reinterpret_cast<WsHeader *>(p.ws);
     uint8_t *records = reinterpret_cast<uint8_t *>(p.ws) + kHeaderBytes;
@@ -548,7 +549,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             st_shared_v4(cbase + (c >> 3) * kAtomBytes + n * 128 + (((c & 7) ^ (n & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
         }
-        if (!IS_INT && use_down) {
+        if (!IS_INT && use_down && !CHUNK_TC) {
             // carry operands start as zeros (only 3 of the 16 K-entries of a row are ever written); the other
             // operand is all ones in bf16
             for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 16; e += kThreads) st_shared_v4(smem_u32(down_a) + e * 16, 0u, 0u, 0u, 0u);
@@ -596,6 +597,23 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             }
             // the data operands start as zeros: only the first pieces of a row are ever rewritten
             for (int e = threadIdx.x; e < kStoreGroups * kAtomBytes / 16; e += kThreads) st_shared_v4(smem_u32(chunk_a) + e * 16, 0u, 0u, 0u, 0u);
+            if (!IS_INT && use_down) {
+                // Down-sweep as a product for s < 128 (the paper's B_s: the carry of what precedes a chunk is added to
+                // every element of the chunk by a matrix product).  The data operand holds, per row, the carry of each
+                // of its chunks in three bf16 terms (K index = 3 g + l, like the chunk totals above); this constant
+                // operand (stored K-major: row n = output column n) has ones where the K index belongs to the chunk
+                // of column n, so that accumulator[r][n] += carry[r][chunk of n].
+                for (int e = threadIdx.x; e < kTileCols * 8; e += kThreads) {
+                    const int n = e >> 3, c = e & 7;
+                    uint32_t wd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int k = c * 8 + i;
+                        if (k < 3 * (kTileCols / S) && k / 3 == n / S) wd[i >> 1] |= 0x3F80u << (16 * (i & 1));
+                    }
+                    st_shared_v4(smem_u32(chunk_sel) + n * 128 + ((c ^ (n & 7)) << 4), wd[0], wd[1], wd[2], wd[3]);
+                }
+            }
         }
         fence_proxy_async_smem();
     }
@@ -1176,6 +1194,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
         // there they must also leave the loop together: the outcome of every wait is then voted on by the
         // whole group.  In the default path a warp shares no barrier with the others and votes alone.
         const bool carry_product = !IS_INT && S == 128 && use_down && !level0_only;
+        const bool chunk_down = CHUNK_TC && !IS_INT && use_down && !level0_only;   // the same for s < 128 (needs the chunk product)
         const bool group_meets = carry_product || CHUNK_TC;       // (the chunk product has the same group barrier)
         auto gave_up = [&](bool ok) {
             return group_meets ? named_barrier_or(3 + group, kEpilogueThreads, !ok) : !__all_sync(0xffffffffu, ok);
@@ -1297,6 +1316,44 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 for (int g = 0; g < kChunks; ++g) {
                     if (IS_INT) chunk_carry[g] = res[2 * g] + (res[2 * g + 1] << 7);
                     else chunk_carry[g] = __float_as_uint((__uint_as_float(res[3 * g]) + __uint_as_float(res[3 * g + 1])) + __uint_as_float(res[3 * g + 2]));
+                }
+                if (chunk_down) {
+                    // Paper-faithful down-sweep for s < 128: what precedes each chunk (row base + carry of the chunk)
+                    // is split exactly into three bf16 terms, the terms of the group's 128 rows replace the chunk
+                    // totals in the data operand (its product has completed), and one product with the 0 / 1 selector
+                    // adds every chunk's carry to all elements of that chunk inside the accumulator.
+                    uint32_t cw[12] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int g = 0; g < kChunks; ++g) {
+                        const float v = __uint_as_float(base) + __uint_as_float(chunk_carry[g]);
+                        const uint32_t hi = __float_as_uint(v) & 0xFFFF0000u;
+                        const float r1 = v - __uint_as_float(hi);
+                        const uint32_t mid = __float_as_uint(r1) & 0xFFFF0000u;
+                        const float r2 = r1 - __uint_as_float(mid);
+                        const uint32_t lo = __float_as_uint(r2) & 0xFFFF0000u;
+                        const uint32_t term[3] = {hi >> 16, mid >> 16, lo >> 16};
+#pragma unroll
+                        for (int l = 0; l < 3; ++l) cw[(3 * g + l) >> 1] |= term[l] << (16 * ((3 * g + l) & 1));
+                        chunk_carry[g] = 0u;                                 // it is inside the accumulator from here on
+                    }
+#pragma unroll
+                    for (int c = 0; c < kPiecesUsed; ++c)
+                        st_shared_v4(rowa + ((c ^ (r & 7)) << 4), cw[4 * c], cw[4 * c + 1], cw[4 * c + 2], cw[4 * c + 3]);
+                    fence_proxy_async_smem();
+                    named_barrier_sync(3 + group, kEpilogueThreads);
+                    if (wq == 0 && lane == 0) {
+                        tc_fence_after();
+                        constexpr int kSelSteps = (3 * kChunks + 15) / 16;
+#pragma unroll
+                        for (int kk = 0; kk < kSelSteps; ++kk)
+                            mma_issue<false>(tmem_base + slot * kTileCols, make_smem_desc(ca + kk * 32),
+                                             make_smem_desc(smem_u32(chunk_sel) + kk * 32), make_idesc(2, kTileCols), 1u);
+                        mma_commit(smem_u32(&ctl->down_done[group]));
+                    }
+                    if (gave_up(w.wait(smem_u32(&ctl->down_done[group]), (j / kStoreGroups) & 1))) break;
+                    tc_fence_after();
+                    run = 0;
+                    base = 0;                                                // (prev keeps the row base: the exclusive value of the row's first element)
                 }
             }
             const uint32_t row0 = lt * kTileRows + wq * 32;           // first 128-element row of this warp's part of the tile

@@ -18,7 +18,7 @@ TILE = 128 * 128
 # and the four warps of a store group meet at barriers inside their loops and have to give up together
 CASES = [("i8", 16, 40, 3, 0, 0), ("f16", 128, 12, 0, 0, 0), ("i8", 64, 400, 150, 0, 0),
          ("i8", 16, 40, 3, 1, 0), ("f16", 16, 200, 160, 1, 0), ("f16", 128, 40, 3, 0, 1), ("f16", 128, 300, 149, 1, 1),
-         ("i8", 16, 40, 3, 2, 0), ("f16", 64, 200, 155, 2, 0)]
+         ("i8", 16, 40, 3, 2, 0), ("f16", 64, 200, 155, 2, 0), ("f16", 16, 200, 151, 2, 1)]
 
 
 @pytest.mark.parametrize("dtype,s,tiles,skip,upper,down", CASES)

@@ -283,6 +283,26 @@ def test_down_sweep_as_a_tensor_core_product(runner, dtype):
     assert runner.stats["down_sweep_path"] == 0
 
 
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_down_sweep_as_a_product_per_chunk(runner, dtype):
+    # s < 128: every chunk's carry (row base + what the earlier chunks of the row add up to) is added to the chunk's
+    # elements by one product with a 0 / 1 selector matrix, the paper's B_s; needs the chunk totals as a product
+    # (upper_level_path = 2), from which the carries come
+    from tests.gpu_util import check
+    for n, s in [(TILE, 16), (9 * TILE + 128 * 3 + 5, 64), (400 * TILE + 77, 16), (300 * TILE, 64)]:
+        for exclusive in (False, True):
+            check(runner, gen(dtype, n, 9100 + n % 127), dtype, s, exclusive, upper_level_path=2, down_sweep_path=1)
+            st = runner.stats
+            assert st["down_sweep_path"] == 1 and st["upper_level_path"] == 2
+            assert st["mma_instructions"] == st["tiles"] * (8 + 8 + 8 + 2 + (2 if s == 16 else 1))
+    for s in (16, 64):
+        got = runner.run(np.ones(1 << 22, np.float16), "f16", s, upper_level_path=2, down_sweep_path=1)   # must stay exact
+        assert np.array_equal(got, np.arange(1, (1 << 22) + 1, dtype=np.float32))
+    check(runner, gen(dtype, 32 * 65536, 6).reshape(32, 65536), dtype, 16, upper_level_path=2, down_sweep_path=1)   # batched rows
+    check(runner, gen("i8", 5 * TILE, 4), "i8", 16, upper_level_path=2, down_sweep_path=1)      # integers: no such product
+    assert runner.stats["down_sweep_path"] == 0
+
+
 def test_widening_copy_measuring_aid():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
