@@ -145,7 +145,11 @@ typedef struct {
  * when it scans the tile totals with the library's own scan (tcu_scan_options_t: variant = 1
  * with upper_level_path >= 1) - the size covers every option of tcu_scan_ex, about 40 bytes
  * per 128 x 128-element tile in all.  Never fails; returns a small non-zero size even for
- * empty problems. */
+ * empty problems.
+ * One workspace may serve calls of different sizes, types and kinds, one after the other on a
+ * stream, if it is large enough for each: records are tagged with the number of the launch that
+ * wrote them, and everything else a call keeps in the workspace (row notes, the two-sweep
+ * scratch) is wiped before the call's work on the stream ends. */
 size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s);
 
 /* Clear a workspace (asynchronous memset on `stream`).  Must run once before the first

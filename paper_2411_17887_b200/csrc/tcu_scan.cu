@@ -218,6 +218,9 @@ tcu_status_t scan_totals_by_scan(const Call &c, uint64_t tiles, uint64_t *inner_
     const size_t in_stride = nested_in_stride(tiles), out_stride = nested_out_stride(tiles);
     uint8_t *planes = base, *sums = base + 4 * in_stride, *inner_ws = sums + 4 * out_stride;
     const unsigned blocks = unsigned((tiles + 255) / 256);
+    // The inner scans' header and records lie where an earlier, larger scan on the same workspace may have kept its
+    // records: they are cleared before use.
+    if (cudaMemsetAsync(inner_ws, 0, nested_ws_bytes(tiles), c.stream) != cudaSuccess) return TCU_ERR_CUDA;
     if (is_int) tcu_totals_split_kernel<true><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), planes, uint32_t(in_stride));
     else tcu_totals_split_kernel<false><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), planes, uint32_t(in_stride));
     if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
@@ -235,7 +238,10 @@ tcu_status_t scan_totals_by_scan(const Call &c, uint64_t tiles, uint64_t *inner_
     }
     if (is_int) tcu_totals_combine_kernel<true><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), sums, uint32_t(out_stride));
     else tcu_totals_combine_kernel<false><<<blocks, 256, 0, c.stream>>>(c.d_ws, uint32_t(tiles), sums, uint32_t(out_stride));
-    return cudaGetLastError() == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+    // Whatever is not a record is wiped before the call returns the workspace: a later, larger scan keeps its records
+    // here, and a left-over word must never read as a record of its epoch (zero is the epoch of no launch).
+    return cudaMemsetAsync(base, 0, nested_bytes(tiles), c.stream) == cudaSuccess ? TCU_OK : TCU_ERR_CUDA;
 }
 
 tcu_status_t scan_impl(const Call &c) {
@@ -411,6 +417,10 @@ tcu_status_t scan_impl(const Call &c) {
             else launch(std::false_type{}, std::false_type{});
         }
         if (cudaGetLastError() != cudaSuccess) return TCU_ERR_CUDA;
+        // The row notes are not records: they are wiped before the call returns the workspace, because a later, larger
+        // scan keeps its records where they lie, and a left-over word must never read as a record of its epoch.
+        if (rows128 > 0 && cudaMemsetAsync(seg_flag, 0, seg_workspace_bytes(cols) - seg_flag_offset(cols), stream) != cudaSuccess)
+            return TCU_ERR_CUDA;
     } else if (tail > 0) {   // the last cols % 128 elements of every scan
         const size_t start = size_t(rows128) * kTileCols;
         if (dt == TCU_I8_I32) {

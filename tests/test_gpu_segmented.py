@@ -147,3 +147,72 @@ def test_segmented_argument_checks():
     assert B.tcu_scan_segmented(d, o, 1024, off, 1, 0, 16, 0, ptr, ws_bytes - 64, 0) == B.TCU_ERR_WORKSPACE
     assert B.tcu_scan_segmented(d, o, 0, off, 0, 0, 16, 0, ptr, ws_bytes, 0) == B.TCU_OK
     assert B.tcu_scan_segmented(d, o, 1024, off, 1, 0, 48, 0, ptr, ws_bytes, 0) == B.TCU_ERR_UNSUPPORTED
+
+
+def test_row_notes_of_a_small_segmented_scan_never_read_as_records_of_a_later_larger_scan():
+    # One workspace, sized for the larger problem, is used by a small segmented scan and then by a large plain scan.  The
+    # row notes of the first lie where the second keeps its tile records.  The notes are chosen so that, read as records,
+    # they would carry the epoch of the second launch and the status "inclusive": rows 4i hand on 4 * 2 + 2 = 10 (one
+    # start at column 118 of an all-ones row), rows 4i + 1 hold no start, rows 4i + 2 hand on 28.  The library wipes its
+    # notes before it returns the workspace, so the large scan must come out right.
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    n_small, n_big = 64 * TILE, 3000 * TILE + 77
+    ws_bytes = max(B.tcu_scan_workspace_bytes(1, n_big, 0, 16), B.tcu_scan_segmented_workspace_bytes(n_small, 0, 16))
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+    ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+    big = inputs.int8_uniform(n_big, -127, 127, 5)
+    d_big = torch.from_numpy(big).cuda()
+    want = so.scan(big, "i8")["y32"]
+    rows = n_small // 128
+    starts = np.concatenate([np.arange(0, rows, 4) * 128 + 118, np.arange(2, rows, 4) * 128 + 100])
+    offsets = np.concatenate([[0], np.sort(starts), [n_small]]).astype(np.int64)
+    ones = np.ones(n_small, dtype=np.int8)
+    d_ones = torch.from_numpy(ones).cuda()
+    d_off = torch.from_numpy(offsets).cuda()
+    for trial in range(3):
+        B.check(B.tcu_scan_workspace_init(ptr, ws_bytes, 0))              # epoch 0: the next two launches use epochs 1 and 2
+        o_small = torch.empty(n_small, dtype=torch.int32, device="cuda")
+        B.check(B.tcu_scan_segmented(d_ones, o_small, n_small, d_off, len(offsets) - 1, 0, 16, 0, ptr, ws_bytes, 0))
+        o_big = torch.empty(n_big, dtype=torch.int32, device="cuda")
+        B.check(B.tcu_scan_inclusive(d_big, o_big, n_big, 0, 16, ptr, ws_bytes, 0))
+        B.check(B.tcu_scan_device_status(ptr, 0))
+        compare(o_small.cpu().numpy(), ones, "i8", offsets, False)
+        got = o_big.cpu().numpy()
+        assert np.array_equal(got, want), f"trial {trial}: first mismatch at {int(np.flatnonzero(got != want)[0])}"
+
+
+def test_one_workspace_shared_by_calls_of_every_kind_and_size():
+    # scans of different kinds leave different things in the workspace (records, row notes, the scratch of the two-sweep
+    # variant); whatever order they come in, on one workspace sized for the largest, every result must be right
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from tests.gpu_util import to_device
+    g = inputs.rng(99)
+    n_max = 700 * TILE + 55
+    ws_bytes = max(B.tcu_scan_workspace_bytes(1, n_max, 0, 16), B.tcu_scan_segmented_workspace_bytes(n_max, 0, 16))
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+    ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+    B.check(B.tcu_scan_workspace_init(ptr, ws_bytes, 0))
+    for it in range(48):
+        kind = ["plain", "segmented", "two_sweep_scanned_totals", "plain", "two_sweep"][it % 5]
+        n = int(g.integers(1, n_max)) if it % 3 else int(g.choice([n_max, 148 * TILE, 3 * TILE + 1, 127]))
+        dtype = ["i8", "f16", "bf16"][int(g.integers(0, 3))]
+        s = int(g.choice([16, 64, 128]))
+        exclusive = bool(g.integers(0, 2))
+        x = gen(dtype, n, 1000 + it)
+        d_in = to_device(x, dtype)
+        out = torch.empty(n, dtype=torch.int32 if dtype == "i8" else torch.float32, device="cuda")
+        dt = B.DTYPES[dtype]
+        if kind == "segmented":
+            off = random_offsets(n, int(g.choice([5, 300, 20000])), it)
+            B.check(B.tcu_scan_segmented(d_in, out, n, torch.from_numpy(off).cuda(), len(off) - 1, dt, s, int(exclusive), ptr, ws_bytes, 0))
+        else:
+            off = np.array([0, n], dtype=np.int64)
+            opts = {"two_sweep": dict(variant=1), "two_sweep_scanned_totals": dict(variant=1, upper_level_path=1)}.get(kind, {})
+            B.check(B.tcu_scan_ex(d_in, out, 1, n, dt, s, ptr, ws_bytes, 0, exclusive=int(exclusive), **opts))
+        B.check(B.tcu_scan_device_status(ptr, 0))
+        try:
+            compare(out.cpu().numpy(), x, dtype, off, exclusive)
+        except AssertionError as e:
+            raise AssertionError(f"call {it} ({kind}, n={n}, {dtype}, s={s}, exclusive={exclusive}): {e}")
