@@ -149,7 +149,10 @@ typedef struct {
  * One workspace may serve calls of different sizes, types and kinds, one after the other on a
  * stream, if it is large enough for each: records are tagged with the number of the launch that
  * wrote them, and everything else a call keeps in the workspace (row notes, the two-sweep
- * scratch) is wiped before the call's work on the stream ends. */
+ * scratch) is wiped before the call's work on the stream ends.  Two calls that could run at the
+ * same time on the GPU (different streams, no dependency between them) need a workspace each.
+ * The launch number is a 32-bit count kept in the workspace: clear the workspace again
+ * (tcu_scan_workspace_init) before it has served 2^32 launches. */
 size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s);
 
 /* Clear a workspace (asynchronous memset on `stream`).  Must run once before the first
