@@ -76,7 +76,6 @@ constexpr int kFirstStoreWarp = 4;                                   // carry ad
 constexpr int kFirstTotalsWarp = kFirstStoreWarp + 4 * kStoreGroups; // totals of rows and tile: 4 warps
 constexpr int kFirstLookbackWarp = kFirstTotalsWarp + 4;             // cross-tile look-back (warp 3 is one more)
 constexpr int kThreads = 32 * (kFirstLookbackWarp + kNumLookbackWarps - 1);
-constexpr int kEpochThread = 2 * 32;     // lane 0 of warp 2: reads the epoch of a launch whose CTAs have one tile each
 // The register re-allocation below assumes that the kernel is compiled at 96 registers per thread, which is what
 // 640 threads per CTA give.  With more threads the compiler settles on fewer (80 at 672), and a setmaxnreg.dec to a
 // value above the current allocation is an illegal instruction: do not add warps without redoing the numbers.
@@ -630,14 +629,9 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
     Waiter w{ctl, hdr, p.spin_limit};
     uint32_t first_ticket = 0;                 // (thread 0 only) first tile of this CTA
     uint32_t my_epoch = 0;                     // (thread 0 only) the epoch of this launch
-    // A launch with no more tiles than CTAs hands tile b to CTA b - nothing to claim, no round trip to the workspace
-    // before the first load - and lets a thread that is idle until the tile lands fetch the epoch.  (With several
-    // tiles per CTA the first one is claimed like the others: a CTA that starts late - behind the tail of the
-    // previous kernel, say - must not sit on an early tile.)
-    const bool single_wave = p.tiles_total <= gridDim.x;
-    if (threadIdx.x == 0) stamp(kStampDepsDone);
-    if (threadIdx.x == (single_wave ? kEpochThread : 0)) {
-        first_ticket = single_wave ? 0u : atomicAdd(&hdr->ticket, 1u);
+    if (threadIdx.x == 0) {
+        stamp(kStampDepsDone);
+        first_ticket = atomicAdd(&hdr->ticket, 1u);
         my_epoch = ld_relaxed_u32(&hdr->epoch) + 1;
         ctl->epoch = my_epoch;
         // what precedes the whole scan (continuation of an earlier piece or shard); only single-array calls pass one
@@ -647,7 +641,10 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
 
     // The j-th tile handled by this CTA is number tile_of[j % kTileRing].  Tiles are claimed at run time with a
     // ticket counter in the workspace, in increasing order: whoever holds tile t knows that every tile before t
-    // is held by a CTA that is already running.  When the tiles run out the producer pushes kNumMarkers "no more
+    // is held by a CTA that is already running.  Nothing is assumed about which CTAs of the grid are resident or in
+    // which order they start (a CTA that has not started holds no tile), so a launch that shares the GPU with another
+    // kernel still makes progress; handing tile b to CTA b would save the first ticket's round trip, but not keep that.
+    // When the tiles run out the producer pushes kNumMarkers "no more
     // tiles" markers through the pipeline, so that every role - and each of the look-back warps, which take the
     // tiles in turns - meets one and stops.
     // Sum of the totals of the tiles before `t`, back to the first tile t0 of the scan or to the nearest tile whose
@@ -792,7 +789,7 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
                 if (!w.wait(smem_u32(&ctl->empty[stage]), (u & 1) ^ 1)) break;
                 PROF_ADD(0);
                 uint32_t t = kNoTile;
-                if (markers == 0) t = single_wave ? (j == 0 ? blockIdx.x : kNoTile) : (j == 0 ? first_ticket : atomicAdd(&hdr->ticket, 1u));
+                if (markers == 0) t = (j == 0) ? first_ticket : atomicAdd(&hdr->ticket, 1u);
                 if (t >= p.tiles_total) t = kNoTile;
                 PROF_ADD(1);
                 PROF_INC(3, 1);
@@ -839,7 +836,6 @@ __global__ void __launch_bounds__(kThreads, 1) tcu_scan_kernel(const __grid_cons
             // again (records are compared with the copy of the epoch in shared memory), and the next launch
             // reads them only after this one has completed.  Doing it here, not at the end of the CTA, keeps
             // the round trip of the atomic off the tail of the kernel.
-            if (single_wave && w.wait(smem_u32(&ctl->epoch_ready), 0)) my_epoch = ctl->epoch;
             {
                 const uint32_t arrived = atomicAdd(&hdr->done, 1u);
                 if (arrived == gridDim.x - 1) {
