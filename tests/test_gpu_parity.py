@@ -326,6 +326,40 @@ def test_widening_copy_measuring_aid():
     assert B.tcu_widen_copy(d_in, d_out, 0, 0, 0) == B.TCU_OK
 
 
+def test_two_streams_at_the_same_time_with_a_workspace_each():
+    # two persistent launches share the SMs: neither may depend on CTAs of its own grid that are not resident yet
+    # (tiles are claimed by running CTAs only), and each keeps its carries in its own workspace
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2411_17887_b200 import binding as B
+    from oracle import scan_oracle as so
+    n_max = 600 * TILE + 77
+    x = gen("i8", n_max, 31)
+    want = so.scan(x, "i8")["y32"]
+    d_in = torch.from_numpy(x).cuda()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    spaces = []
+    for _ in streams:
+        ws_bytes = B.tcu_scan_workspace_bytes(1, n_max, 0, 16)
+        ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+        ptr = ws.data_ptr() + (-ws.data_ptr()) % 256
+        B.check(B.tcu_scan_workspace_init(ptr, ws_bytes, 0))
+        spaces.append((ws, ptr, ws_bytes))
+    torch.cuda.synchronize()
+    results = []
+    for n, s in [(n_max, 16), (148 * TILE, 64), (100 * TILE + 5, 128), (n_max, 64), (TILE, 16), (300 * TILE, 16)]:
+        for strm, (ws, ptr, ws_bytes) in zip(streams, spaces):
+            with torch.cuda.stream(strm):
+                out = torch.empty(n, dtype=torch.int32, device="cuda")
+                B.check(B.tcu_scan_inclusive(d_in, out, n, 0, s, ptr, ws_bytes, strm.cuda_stream))
+                results.append((n, out))
+    torch.cuda.synchronize()
+    for ws, ptr, ws_bytes in spaces:
+        assert B.tcu_scan_device_status(ptr, 0) == B.TCU_OK
+    for n, out in results:
+        assert np.array_equal(out.cpu().numpy(), want[:n])
+
+
 def test_many_back_to_back_launches_agree(runner):
     # consecutive launches overlap their set-up with the previous kernel's tail and reuse one workspace:
     # every one of them must reproduce the integers of the first, whatever the number of CTAs
