@@ -163,7 +163,7 @@ tcu_status_t tcu_scan_workspace_init(void *d_ws, size_t ws_bytes, cudaStream_t s
  * "prefix sum"; Algorithm 1 + Section 2.2 for arbitrary n).
  *   d_in   device, n elements of the input type, 16-byte aligned
  *   d_out  device, n elements of the output type (4 bytes each), 16-byte aligned
- *   n      any value >= 0 (n = 0 returns TCU_OK without a launch)
+ *   n      any value from 0 to 2^37 (n = 0 returns TCU_OK without a launch; more: TCU_ERR_UNSUPPORTED)
  *   d_ws   device workspace of at least tcu_scan_workspace_bytes(1, n, dt, s) bytes */
 tcu_status_t tcu_scan_inclusive(const void *d_in, void *d_out, size_t n, tcu_dtype_t dt, int s,
                                 void *d_ws, size_t ws_bytes, cudaStream_t stream);
@@ -178,7 +178,7 @@ tcu_status_t tcu_scan_exclusive(const void *d_in, void *d_out, size_t n, tcu_dty
  * (Section 2.2 step 1: the algorithm run on each contiguous segment, no stitching).
  * Any cols >= 1.  When cols is a multiple of 16 every row starts 16-byte aligned and the rows
  * are tiled one by one; otherwise the array is tiled as a whole and the row starts are
- * segment boundaries inside it (the path of tcu_scan_segmented; rows * cols < 2^40).
+ * segment boundaries inside it (the path of tcu_scan_segmented; rows * cols <= 2^37).
  *   d_ws   at least tcu_scan_workspace_bytes(rows, cols, dt, s) bytes */
 tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t cols,
                               tcu_dtype_t dt, int s, int exclusive,

@@ -41,6 +41,8 @@ int elem_bytes(tcu_dtype_t dt) { return dt == TCU_I8_I32 ? 1 : 2; }
 bool valid_dtype(int dt) { return dt == TCU_I8_I32 || dt == TCU_F16_F32 || dt == TCU_BF16_F32; }
 bool valid_s(int s) { return s == 16 || s == 64 || s == 128; }
 
+constexpr uint64_t kMaxScanElements = 1ull << 37;       // elements of one scan (one row): 2^30 rows of 128
+
 uint64_t tiles_for(uint64_t rows, uint64_t cols) {
     uint64_t rows128 = cols / kTileCols;                       // full 128-element rows of one scan
     uint64_t per = (rows128 + kTileRows - 1) / kTileRows;      // tiles of one scan
@@ -181,7 +183,8 @@ tcu_status_t check_call(const Call &c) {
     // dense rows: the row pitch must keep every row 16-byte aligned on both sides (TMA boxes, vector stores)
     if (c.rows > 1 && ((c.cols * eb) % 16 != 0 || (c.cols * 4) % 16 != 0)) return TCU_ERR_UNSUPPORTED;
     if (c.level0 && (c.cols % kTileCols) != 0) return TCU_ERR_UNSUPPORTED;
-    if (c.rows > (1ull << 31) || c.cols > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
+    // (a scan is addressed by TMA as rows of 128 elements with a 32-bit signed row coordinate)
+    if (c.rows > (1ull << 31) || c.cols > kMaxScanElements) return TCU_ERR_UNSUPPORTED;
     if (c.rows > 1 && (c.d_carry_in || c.d_carry_out)) return TCU_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(c.d_carry_in) & 7) || (reinterpret_cast<uintptr_t>(c.d_carry_out) & 7)) return TCU_ERR_INVALID_ARG;
     if (c.two_sweep && (c.rows > 1 || c.d_carry_in || c.d_carry_out)) return TCU_ERR_UNSUPPORTED;
@@ -544,7 +547,7 @@ tcu_status_t tcu_scan_batched(const void *d_in, void *d_out, size_t rows, size_t
     if (rows > 1 && cols % 16 != 0) {
         // rows that do not start 16-byte aligned cannot be tiled one by one: tile the array as a whole and treat
         // the row starts as segment starts
-        if (cols > (1ull << 40) / rows) return TCU_ERR_UNSUPPORTED;
+        if (cols > kMaxScanElements / rows) return TCU_ERR_UNSUPPORTED;
         Call c = make_call(d_in, d_out, 1, rows * cols, dt, s, exclusive != 0, d_ws, ws_bytes, stream);
         c.segmented = true;
         c.seg_pitch = cols;
@@ -707,7 +710,7 @@ tcu_status_t tcu_reduce_total(const void *d_in, size_t n, tcu_dtype_t dt, void *
     if (!valid_dtype(dt)) return TCU_ERR_INVALID_ARG;
     if (!d_total || (reinterpret_cast<uintptr_t>(d_total) & 7)) return TCU_ERR_INVALID_ARG;
     if (n > 0 && (!d_in || (reinterpret_cast<uintptr_t>(d_in) & 15))) return TCU_ERR_INVALID_ARG;
-    if (n > (1ull << 40)) return TCU_ERR_UNSUPPORTED;
+    if (n > kMaxScanElements) return TCU_ERR_UNSUPPORTED;
     if (!d_ws) return TCU_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(d_ws) & 255) return TCU_ERR_INVALID_ARG;
     if (ws_bytes < tcu_scan_workspace_bytes(1, n + kTileElems, dt, 16)) return TCU_ERR_WORKSPACE;

@@ -77,6 +77,10 @@ def test_argument_checks_return_before_any_launch(B):
     assert B.tcu_scan_exclusive(ok_in, ok_out, 1 << 20, 0, 16, ok_ws, 64) == B.TCU_ERR_WORKSPACE    # too small
     assert B.tcu_scan_inclusive(ok_in, ok_in + 64, 1 << 10, 0, 16, ok_ws, ws) == B.TCU_ERR_INVALID_ARG  # overlap
     assert B.tcu_scan_batched(ok_in, ok_out, 4, (1 << 40) + 16, 0, 16, 0, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED   # too large
+    # one scan holds at most 2^37 elements (2^30 rows of 128 under a signed 32-bit row coordinate)
+    far_in, far_out = 0x10000, 0x7000_0000_0000
+    assert B.tcu_scan_inclusive(far_in, far_out, (1 << 37) + 128, 0, 16, ok_ws, ws) == B.TCU_ERR_UNSUPPORTED
+    assert B.tcu_scan_inclusive(far_in, far_out, 1 << 37, 0, 16, ok_ws, ws) == B.TCU_ERR_WORKSPACE       # the size itself is accepted
     # the general call: malformed options are refused, carries belong to single arrays only
     assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, variant=2) == B.TCU_ERR_INVALID_ARG
     assert B.tcu_scan_ex(ok_in, ok_out, 1, 10, 0, 16, ok_ws, ws, upper_level_path=3) == B.TCU_ERR_INVALID_ARG
