@@ -152,7 +152,10 @@ typedef struct {
  * scratch) is wiped before the call's work on the stream ends.  Two calls that could run at the
  * same time on the GPU (different streams, no dependency between them) need a workspace each.
  * The launch number is a 32-bit count kept in the workspace: clear the workspace again
- * (tcu_scan_workspace_init) before it has served 2^32 launches. */
+ * (tcu_scan_workspace_init) before it has served 2^32 launches.
+ * The scan calls that take a workspace only queue kernels and memsets on `stream` (no
+ * synchronisation, no allocation), so a sequence of them can be captured into a CUDA graph and
+ * replayed (tested for tcu_scan_inclusive). */
 size_t tcu_scan_workspace_bytes(size_t rows, size_t cols, tcu_dtype_t dt, int s);
 
 /* Clear a workspace (asynchronous memset on `stream`).  Must run once before the first

@@ -360,6 +360,32 @@ def test_two_streams_at_the_same_time_with_a_workspace_each():
         assert np.array_equal(out.cpu().numpy(), want[:n])
 
 
+def test_scans_replayed_from_a_cuda_graph(runner):
+    # the workspace entry points only queue work on the given stream (kernels, and memsets for the segmented path), so a
+    # sequence of scans can be captured once and replayed; every replay must give the same integers as the oracle
+    from paper_2411_17887_b200 import binding as B
+    from oracle import scan_oracle as so
+    sizes = [(1 << 16, 16), (37 * TILE + 128 * 5 + 9, 64), (300 * TILE + 77, 16)]
+    xs = [gen("i8", n, 600 + i) for i, (n, s) in enumerate(sizes)]
+    d_ins = [torch.from_numpy(x).cuda() for x in xs]
+    outs = [torch.zeros(x.size, dtype=torch.int32, device="cuda") for x in xs]
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        cap = torch.cuda.current_stream().cuda_stream
+        for (n, s), d_in, out in zip(sizes, d_ins, outs):
+            B.check(B.tcu_scan_inclusive(d_in, out, n, 0, s, runner.ws_ptr, runner.ws_bytes, cap))
+    for replay in range(3):
+        for out in outs:
+            out.fill_(-1)
+        graph.replay()
+        torch.cuda.synchronize()
+        B.check(B.tcu_scan_device_status(runner.ws_ptr, 0))
+        for x, out in zip(xs, outs):
+            assert np.array_equal(out.cpu().numpy(), so.scan(x, "i8")["y32"]), f"replay {replay}"
+    del graph
+
+
 def test_many_back_to_back_launches_agree(runner):
     # consecutive launches overlap their set-up with the previous kernel's tail and reuse one workspace:
     # every one of them must reproduce the integers of the first, whatever the number of CTAs
